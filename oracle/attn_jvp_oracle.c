@@ -1,0 +1,319 @@
+/*
+ * attn_jvp_oracle.c -- TEST INFRASTRUCTURE, not part of the product path.
+ *
+ * Plain fp64 CPU oracle for the forward-mode Jacobian-vector product (JVP) of
+ * non-causal softmax attention (Appendix C.1, "FlashAttention-2 JVP").
+ * Only the tests, the smoke check and the benchmark's cpu_baseline / reference
+ * leg may build, load or call this file.  It shares no code with the CUDA path.
+ *
+ * Two independent routes to the same numbers live here:
+ *
+ *   attn_jvp_def_*   the definition written out row by row (the unnumbered
+ *                    equations of Appendix C.1: S, P = softmax(S), O = P V,
+ *                    tS = tQ K^T + Q tK^T, tP = P.tS - P.(rowsum(P.tS) 1 1^T),
+ *                    tO = tP V + P tV), two passes over one row of scores.
+ *
+ *   attn_jvp_alg2_*  the streaming procedure of Algorithm 2 taken step by step
+ *                    in the paper's order and notation (m, l, r, O, A, B per
+ *                    query row, key blocks of size B_c, epilogue O/l, L = m +
+ *                    log l, C = r O, tO = (A + B - C)/l).
+ *
+ * Readings where the paper is silent:
+ *   - the paper writes S = Q K^T with no softmax scale; here S = s Q K^T and
+ *     tS = s (tQ K^T + Q tK^T) with a constant s ("scale");
+ *   - L (the log-sum-exp) is the natural log of sum_j exp(S_ij);
+ *   - the (P.tS) 1 1^T term is the per-row scalar mu_i = sum_j P_ij tS_ij
+ *     broadcast along the row; mu is returned as an extra output because
+ *     d(LSE_i) = mu_i, which gives a second finite-difference pin.
+ *
+ * Pins (tests/, "not gpu"): central finite differences of O and LSE, linearity
+ * in the tangent, zero tangent, Lk = 1, Q = 0 closed form, constant-V,
+ * hand-derived golden values, torch.func.jvp, and def == alg2 on brute-force
+ * tiny shapes.
+ *
+ * All matrices handed to the *_f64 entry points are dense row-major doubles:
+ * Q,tQ [Lq][D]; K,tK,V,tV [Lk][D]; O,tO [Lq][D]; LSE,mu [Lq].
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ------------------------------------------------------------------------- */
+/* One query row, by the definition.  s_buf and ts_buf hold Lk doubles each. */
+static void def_row(const double *q, const double *tq,
+                    const double *K, const double *tK,
+                    const double *V, const double *tV,
+                    long Lk, long D, long ldk, double scale,
+                    double *o, double *to, double *lse, double *mu,
+                    double *s_buf, double *ts_buf)
+{
+    /* S_ij = s * sum_d Q_id K_jd ;  tS_ij = s * sum_d (tQ_id K_jd + Q_id tK_jd) */
+    double m = -INFINITY;
+    for (long j = 0; j < Lk; ++j) {
+        const double *kj = K + j * ldk;
+        double s = 0.0, ts = 0.0;
+        for (long d = 0; d < D; ++d) {
+            s += q[d] * kj[d];
+            ts += tq[d] * kj[d];
+        }
+        if (tK) {
+            const double *tkj = tK + j * ldk;
+            for (long d = 0; d < D; ++d) ts += q[d] * tkj[d];
+        }
+        s_buf[j] = scale * s;
+        ts_buf[j] = scale * ts;
+        if (s_buf[j] > m) m = s_buf[j];
+    }
+    /* P_ij = exp(S_ij - m_i) / sum_j exp(S_ij - m_i) */
+    double denom = 0.0;
+    for (long j = 0; j < Lk; ++j) {
+        s_buf[j] = exp(s_buf[j] - m);
+        denom += s_buf[j];
+    }
+    for (long j = 0; j < Lk; ++j) s_buf[j] /= denom;
+    /* mu_i = sum_j P_ij tS_ij  (the rowsum(P.tS) term) */
+    double mu_i = 0.0;
+    for (long j = 0; j < Lk; ++j) mu_i += s_buf[j] * ts_buf[j];
+    /* O_i = sum_j P_ij V_j ; tO_i = sum_j tP_ij V_j + sum_j P_ij tV_j,
+       tP_ij = P_ij tS_ij - P_ij mu_i */
+    for (long d = 0; d < D; ++d) { o[d] = 0.0; to[d] = 0.0; }
+    for (long j = 0; j < Lk; ++j) {
+        const double p = s_buf[j];
+        const double tp = p * ts_buf[j] - p * mu_i;
+        const double *vj = V + j * ldk;
+        for (long d = 0; d < D; ++d) {
+            o[d] += p * vj[d];
+            to[d] += tp * vj[d];
+        }
+        if (tV) {
+            const double *tvj = tV + j * ldk;
+            for (long d = 0; d < D; ++d) to[d] += p * tvj[d];
+        }
+    }
+    *lse = m + log(denom);
+    *mu = mu_i;
+}
+
+/* Definition route, fp64 in / fp64 out.  tK and tV may be NULL (zero tangent). */
+int attn_jvp_def_f64(const double *Q, const double *K, const double *V,
+                     const double *tQ, const double *tK, const double *tV,
+                     long Lq, long Lk, long D, double scale,
+                     double *O, double *tO, double *LSE, double *MU)
+{
+    if (Lq < 1 || Lk < 1 || D < 1) return 1;
+    int fail = 0;
+#pragma omp parallel
+    {
+        double *s_buf = (double *)malloc(sizeof(double) * (size_t)Lk);
+        double *ts_buf = (double *)malloc(sizeof(double) * (size_t)Lk);
+        if (!s_buf || !ts_buf) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp barrier
+        if (!fail) {
+#pragma omp for schedule(dynamic, 4)
+            for (long i = 0; i < Lq; ++i)
+                def_row(Q + i * D, tQ + i * D, K, tK, V, tV, Lk, D, D, scale,
+                        O + i * D, tO + i * D, LSE + i, MU + i, s_buf, ts_buf);
+        }
+        free(s_buf);
+        free(ts_buf);
+    }
+    return fail ? 2 : 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Algorithm 2, one query row (B_r = 1; rows never interact), key blocks B_c. */
+static void alg2_row(const double *q, const double *tq,
+                     const double *K, const double *tK,
+                     const double *V, const double *tV,
+                     long Lk, long D, long Bc, double scale,
+                     double *o_out, double *to_out, double *lse, double *mu,
+                     double *work /* 3*D + 2*Bc doubles */)
+{
+    double *Oi = work, *Ai = work + D, *Bi = work + 2 * D;
+    double *Pt = work + 3 * D, *tSij = Pt + Bc;
+    /* initialise m = -inf, l = 0, O = 0, r = 0, A = 0, B = 0 */
+    double m_i = -INFINITY, l_i = 0.0, r_i = 0.0;
+    for (long d = 0; d < D; ++d) { Oi[d] = 0.0; Ai[d] = 0.0; Bi[d] = 0.0; }
+
+    for (long j0 = 0; j0 < Lk; j0 += Bc) {
+        const long nb = (Lk - j0 < Bc) ? (Lk - j0) : Bc;
+        /* S_ij = Q_i K_j^T ; tS_ij = tQ_i K_j^T + Q_i tK_j^T */
+        double rowmax = -INFINITY;
+        for (long c = 0; c < nb; ++c) {
+            const double *kj = K + (j0 + c) * D;
+            double s = 0.0, ts = 0.0;
+            for (long d = 0; d < D; ++d) { s += q[d] * kj[d]; ts += tq[d] * kj[d]; }
+            if (tK) {
+                const double *tkj = tK + (j0 + c) * D;
+                for (long d = 0; d < D; ++d) ts += q[d] * tkj[d];
+            }
+            Pt[c] = scale * s;
+            tSij[c] = scale * ts;
+            if (Pt[c] > rowmax) rowmax = Pt[c];
+        }
+        /* m_new = max(m_i, rowmax(S_ij)) */
+        const double m_new = (m_i > rowmax) ? m_i : rowmax;
+        /* P~_ij = exp(S_ij - m_new) */
+        double rowsum_P = 0.0;
+        for (long c = 0; c < nb; ++c) { Pt[c] = exp(Pt[c] - m_new); rowsum_P += Pt[c]; }
+        const double alpha = exp(m_i - m_new); /* e^{m_i - m_new}; 0 on the first block */
+        /* l_new = alpha l_i + rowsum(P~) */
+        const double l_new = alpha * l_i + rowsum_P;
+        /* O_new = alpha O_i + P~ V_j ; A_new = alpha A_i + P~ tV_j */
+        for (long d = 0; d < D; ++d) { Oi[d] *= alpha; Ai[d] *= alpha; Bi[d] *= alpha; }
+        for (long c = 0; c < nb; ++c) {
+            const double *vj = V + (j0 + c) * D;
+            for (long d = 0; d < D; ++d) Oi[d] += Pt[c] * vj[d];
+            if (tV) {
+                const double *tvj = tV + (j0 + c) * D;
+                for (long d = 0; d < D; ++d) Ai[d] += Pt[c] * tvj[d];
+            }
+        }
+        /* H~_ij = P~_ij . tS_ij ; r_new = alpha r_i + rowsum(H~) ; B_new = alpha B_i + H~ V_j */
+        double rowsum_H = 0.0;
+        for (long c = 0; c < nb; ++c) {
+            const double h = Pt[c] * tSij[c];
+            rowsum_H += h;
+            const double *vj = V + (j0 + c) * D;
+            for (long d = 0; d < D; ++d) Bi[d] += h * vj[d];
+        }
+        const double r_new = alpha * r_i + rowsum_H;
+        m_i = m_new; l_i = l_new; r_i = r_new;
+    }
+    /* O_i = O/l ; L_i = m + log l ; C_i = r O_i ; tO_i = (A + B - C)/l */
+    for (long d = 0; d < D; ++d) o_out[d] = Oi[d] / l_i;
+    *lse = m_i + log(l_i);
+    for (long d = 0; d < D; ++d) {
+        const double Cd = r_i * o_out[d];
+        to_out[d] = (Ai[d] + Bi[d] - Cd) / l_i;
+    }
+    *mu = r_i / l_i;
+}
+
+int attn_jvp_alg2_f64(const double *Q, const double *K, const double *V,
+                      const double *tQ, const double *tK, const double *tV,
+                      long Lq, long Lk, long D, long Bc, double scale,
+                      double *O, double *tO, double *LSE, double *MU)
+{
+    if (Lq < 1 || Lk < 1 || D < 1 || Bc < 1) return 1;
+    int fail = 0;
+#pragma omp parallel
+    {
+        double *work = (double *)malloc(sizeof(double) * (size_t)(3 * D + 2 * Bc));
+        if (!work) {
+#pragma omp atomic write
+            fail = 1;
+        }
+#pragma omp barrier
+        if (!fail) {
+#pragma omp for schedule(dynamic, 4)
+            for (long i = 0; i < Lq; ++i)
+                alg2_row(Q + i * D, tQ + i * D, K, tK, V, tV, Lk, D, Bc, scale,
+                         O + i * D, tO + i * D, LSE + i, MU + i, work);
+        }
+        free(work);
+    }
+    return fail ? 2 : 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/* bf16 bit patterns, [B][L][H][D] ("BLHD") layout, selected rows.           */
+
+static double bf16_to_f64(uint16_t h)
+{
+    uint32_t u = ((uint32_t)h) << 16; /* bf16 is the top half of an fp32 */
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* Widen one head's [L][D] slice out of a BLHD bf16 tensor. */
+static void widen_head(const uint16_t *x, long b, long h, long L, long H, long D, double *dst)
+{
+    for (long l = 0; l < L; ++l) {
+        const uint16_t *src = x + ((b * L + l) * H + h) * D;
+        for (long d = 0; d < D; ++d) dst[l * D + d] = bf16_to_f64(src[d]);
+    }
+}
+
+/*
+ * Definition route on bf16 BLHD inputs for a list of query rows.
+ * rows[n] is a flat index (b*H + h)*Lq + i, sorted so that equal (b,h) are
+ * adjacent (the head's K/V are widened once per run of equal heads).
+ * Outputs: O,tO [nrows][D]; LSE,MU [nrows] in fp64.
+ * tk / tv may be NULL (cross-attention with a constant context: tK = tV = 0).
+ */
+int attn_jvp_def_bf16_blhd_rows(const uint16_t *q, const uint16_t *k, const uint16_t *v,
+                                const uint16_t *tq, const uint16_t *tk, const uint16_t *tv,
+                                long B, long H, long Lq, long Lk, long D, double scale,
+                                const int64_t *rows, long nrows,
+                                double *O, double *tO, double *LSE, double *MU)
+{
+    if (B < 1 || H < 1 || Lq < 1 || Lk < 1 || D < 1 || nrows < 0) return 1;
+    const size_t kv = (size_t)Lk * (size_t)D;
+    double *Kd = (double *)malloc(sizeof(double) * kv);
+    double *Vd = (double *)malloc(sizeof(double) * kv);
+    double *tKd = tk ? (double *)malloc(sizeof(double) * kv) : NULL;
+    double *tVd = tv ? (double *)malloc(sizeof(double) * kv) : NULL;
+    int rc = 0;
+    if (!Kd || !Vd || (tk && !tKd) || (tv && !tVd)) rc = 2;
+
+    long n0 = 0;
+    while (rc == 0 && n0 < nrows) {
+        const long bh = (long)(rows[n0] / Lq);
+        long n1 = n0;
+        while (n1 < nrows && (long)(rows[n1] / Lq) == bh) ++n1;
+        if (bh < 0 || bh >= B * H) { rc = 3; break; }
+        const long b = bh / H, h = bh % H;
+        widen_head(k, b, h, Lk, H, D, Kd);
+        widen_head(v, b, h, Lk, H, D, Vd);
+        if (tk) widen_head(tk, b, h, Lk, H, D, tKd);
+        if (tv) widen_head(tv, b, h, Lk, H, D, tVd);
+#pragma omp parallel
+        {
+            double *s_buf = (double *)malloc(sizeof(double) * (size_t)Lk);
+            double *ts_buf = (double *)malloc(sizeof(double) * (size_t)Lk);
+            double *qd = (double *)malloc(sizeof(double) * (size_t)D * 2);
+            if (!s_buf || !ts_buf || !qd) {
+#pragma omp atomic write
+                rc = 2;
+            }
+#pragma omp barrier
+            if (rc == 0) {
+#pragma omp for schedule(dynamic, 4)
+                for (long n = n0; n < n1; ++n) {
+                    const long i = (long)(rows[n] % Lq);
+                    const uint16_t *qs = q + ((b * Lq + i) * H + h) * D;
+                    const uint16_t *tqs = tq + ((b * Lq + i) * H + h) * D;
+                    for (long d = 0; d < D; ++d) {
+                        qd[d] = bf16_to_f64(qs[d]);
+                        qd[D + d] = bf16_to_f64(tqs[d]);
+                    }
+                    def_row(qd, qd + D, Kd, tKd, Vd, tVd, Lk, D, D, scale,
+                            O + n * D, tO + n * D, LSE + n, MU + n, s_buf, ts_buf);
+                }
+            }
+            free(s_buf); free(ts_buf); free(qd);
+        }
+        n0 = n1;
+    }
+    free(Kd); free(Vd); free(tKd); free(tVd);
+    return rc;
+}
+
+int attn_jvp_oracle_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
