@@ -1,0 +1,109 @@
+/*
+ * attn_jvp.h -- C ABI of the B200 (sm_100a) attention-JVP library.
+ *
+ * One operation: the forward-mode Jacobian-vector product of non-causal
+ * softmax attention, fused into a single streaming pass over the keys
+ * (Appendix C.1 "FlashAttention-2 JVP", Algorithm 2).  For every batch b and
+ * head h independently, with s = `scale`:
+ *
+ *     S  = s Q K^T                P  = softmax_rows(S)          O = P V
+ *     tS = s (tQ K^T + Q tK^T)    mu = rowsum(P . tS)
+ *     tO = (P . tS) V + P tV - diag(mu) O                       (aggregated form, Appendix C.1)
+ *     LSE_i = log sum_j exp(S_ij)                               (Algorithm 2, L = m + log l)
+ *
+ * The paper writes S = Q K^T without a softmax scale; here the constant
+ * `scale` multiplies both S and tS and is not differentiated.
+ *
+ * Conventions common to every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller.  The
+ *     library neither frees nor retains them, allocates no device memory and
+ *     needs no workspace.
+ *   - q, tq, o, to : bf16, layout [B][Lq][H][D] contiguous ("BLHD").
+ *     k, v, tk, tv : bf16, layout [B][Lk][H][D] contiguous.
+ *     lse          : fp32, layout [B][H][Lq], natural log of the scaled scores.
+ *   - D is 64 or 128.  Lq and Lk are arbitrary positive lengths (no multiple
+ *     of the tile size is required).  Same H for queries and keys.
+ *   - Arithmetic: bf16 operands, fp32 accumulation, outputs rounded to bf16
+ *     (round to nearest even).  Inputs are assumed finite.
+ *   - Calls are asynchronous: work is enqueued on a CUDA stream and the
+ *     function returns.  Rows i >= Lq are never written.
+ *   - Return value: 0 on success, otherwise one of the ATTN_JVP_ERR_* codes
+ *     below, in which case NOTHING has been enqueued.  No exceptions, no
+ *     exit(), no CPU fallback.
+ *   - Every device-side wait is bounded.  If one expires (a bug, never expected)
+ *     the kernel stops early and records ATTN_JVP_ERR_DEVICE_TIMEOUT, which
+ *     attn_jvp_device_status() reports after the caller has synchronised.
+ */
+#ifndef ATTN_JVP_H_
+#define ATTN_JVP_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* flags */
+#define ATTN_JVP_KV_TANGENT_FREE 0x1u /* tK = tV = 0 (cross-attention on a constant context,  */
+                                      /* Sec. 3.2 / Appendix C.2); tk, tv ignored, may be NULL */
+#define ATTN_JVP_FWD_ONLY        0x2u /* plain forward of the same kernel: only O and LSE are  */
+                                      /* produced; tq, tk, tv, to ignored, may be NULL         */
+
+/* error codes */
+#define ATTN_JVP_OK                  0
+#define ATTN_JVP_ERR_NULL            1  /* a required pointer is NULL */
+#define ATTN_JVP_ERR_SHAPE           2  /* B, H, Lq or Lk < 1, or sizes overflow */
+#define ATTN_JVP_ERR_UNSUPPORTED_D   3  /* D is not 64 or 128 */
+#define ATTN_JVP_ERR_ALIGN           4  /* a tensor pointer is not 16-byte aligned */
+#define ATTN_JVP_ERR_FLAGS           5  /* unknown flag bits */
+#define ATTN_JVP_ERR_SCALE           6  /* scale is NaN or infinite */
+#define ATTN_JVP_ERR_ALIAS           7  /* an output buffer overlaps an input or another output */
+#define ATTN_JVP_ERR_ARCH            8  /* current device is not compute capability 10.x */
+#define ATTN_JVP_ERR_CUDA            9  /* a CUDA runtime / driver call failed (see strerror) */
+#define ATTN_JVP_ERR_DEVICE_TIMEOUT 10  /* a bounded device-side wait expired */
+
+/*
+ * attn_jvp_fwd -- O, tO and LSE of Algorithm 2 in one pass, on the stream set
+ * by attn_jvp_set_stream (default: the legacy default stream).
+ *
+ *   q,k,v,tq,tk,tv  inputs (device, bf16 BLHD).  With ATTN_JVP_KV_TANGENT_FREE
+ *                   tk and tv are not read.  With ATTN_JVP_FWD_ONLY tq, tk, tv
+ *                   are not read and `to` is not written.
+ *   o, to           outputs (device, bf16 BLHD, [B][Lq][H][D]).
+ *   lse             output (device, fp32 [B][H][Lq]).
+ *   B,H,Lq,Lk,D     sizes; scale: softmax scale s; flags: ATTN_JVP_* bits.
+ */
+int attn_jvp_fwd(const void* q, const void* k, const void* v,
+                 const void* tq, const void* tk, const void* tv,
+                 void* o, void* to, float* lse,
+                 int B, int H, int Lq, int Lk, int D,
+                 float scale, unsigned flags);
+
+/* Same operation (Algorithm 2) on an explicit CUDA stream (a cudaStream_t passed as void*). */
+int attn_jvp_fwd_stream(const void* q, const void* k, const void* v,
+                        const void* tq, const void* tk, const void* tv,
+                        void* o, void* to, float* lse,
+                        int B, int H, int Lq, int Lk, int D,
+                        float scale, unsigned flags, void* cuda_stream);
+
+/* Sets the stream attn_jvp_fwd launches on for the calling host thread
+ * (thread-local; NULL = legacy default stream).  Always returns 0. */
+int attn_jvp_set_stream(void* cuda_stream);
+
+/*
+ * Device-side status of the current device since the last call of this
+ * function: 0, or ATTN_JVP_ERR_DEVICE_TIMEOUT if a bounded wait inside a
+ * kernel expired.  Meaningful once the caller has synchronised the stream(s)
+ * the kernels ran on; reading it clears it.  Does not synchronise.
+ */
+int attn_jvp_device_status(void);
+
+/* Human-readable text for a return code; for ATTN_JVP_ERR_CUDA the text of the
+ * last failing CUDA call on this thread is appended.  Never NULL. */
+const char* attn_jvp_strerror(int code);
+
+/* Library version: major*10000 + minor*100 + patch. */
+int attn_jvp_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ATTN_JVP_H_ */

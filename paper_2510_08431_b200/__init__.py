@@ -1,0 +1,5 @@
+"""B200 (sm_100a) attention-JVP library: Python binding of the C ABI in include/attn_jvp.h."""
+from . import synth  # noqa: F401
+from .attn_jvp import (  # noqa: F401
+    FWD_ONLY, KV_TANGENT_FREE, AttnJvpError, attention_jvp, attention_jvp_host, attn_jvp_device_status,
+    attn_jvp_fwd, attn_jvp_fwd_stream, attn_jvp_set_stream, attn_jvp_strerror, attn_jvp_version, load)

@@ -1,0 +1,158 @@
+"""Thin Python binding of the C ABI in include/attn_jvp.h (argument marshalling only).
+
+Every step of the computation runs inside the CUDA library; PyTorch is used for
+device memory and streams.  There is no CPU or eager fallback: if the library is
+missing or the device is not sm_100, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+import threading
+
+import torch
+
+KV_TANGENT_FREE = 0x1
+FWD_ONLY = 0x2
+
+ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED_D, ERR_ALIGN, ERR_FLAGS = 1, 2, 3, 4, 5
+ERR_SCALE, ERR_ALIAS, ERR_ARCH, ERR_CUDA, ERR_DEVICE_TIMEOUT = 6, 7, 8, 9, 10
+
+EXPORTS = ("attn_jvp_fwd", "attn_jvp_fwd_stream", "attn_jvp_set_stream", "attn_jvp_device_status",
+           "attn_jvp_strerror", "attn_jvp_version")
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libattn_jvp.so")
+_lock = threading.Lock()
+_lib = None
+
+
+class AttnJvpError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"attn_jvp error {code}: {msg}")
+        self.code = code
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load():
+    """Loads libattn_jvp.so (built in-tree by paper_2510_08431_b200.build); raises if it is missing."""
+    global _lib
+    with _lock:
+        if _lib is None:
+            if not os.path.exists(_LIB_PATH):
+                raise RuntimeError(
+                    f"{_LIB_PATH} is missing: build it with `python -m paper_2510_08431_b200.build` "
+                    "(there is no fallback path)")
+            lib = ctypes.CDLL(_LIB_PATH)
+            vp, ci, cu, cf = ctypes.c_void_p, ctypes.c_int, ctypes.c_uint, ctypes.c_float
+            common = [vp] * 9 + [ci] * 5 + [cf, cu]
+            lib.attn_jvp_fwd.argtypes = common
+            lib.attn_jvp_fwd.restype = ci
+            lib.attn_jvp_fwd_stream.argtypes = common + [vp]
+            lib.attn_jvp_fwd_stream.restype = ci
+            lib.attn_jvp_set_stream.argtypes = [vp]
+            lib.attn_jvp_set_stream.restype = ci
+            lib.attn_jvp_device_status.argtypes = []
+            lib.attn_jvp_device_status.restype = ci
+            lib.attn_jvp_strerror.argtypes = [ci]
+            lib.attn_jvp_strerror.restype = ctypes.c_char_p
+            lib.attn_jvp_version.argtypes = []
+            lib.attn_jvp_version.restype = ci
+            _lib = lib
+    return _lib
+
+
+def _ptr(x):
+    if x is None:
+        return None
+    if isinstance(x, torch.Tensor):
+        return x.data_ptr()
+    return int(x)
+
+
+def attn_jvp_strerror(code: int) -> str:
+    return load().attn_jvp_strerror(int(code)).decode()
+
+
+def attn_jvp_version() -> int:
+    return int(load().attn_jvp_version())
+
+
+def attn_jvp_set_stream(cuda_stream) -> int:
+    return int(load().attn_jvp_set_stream(_ptr(cuda_stream)))
+
+
+def attn_jvp_device_status() -> int:
+    return int(load().attn_jvp_device_status())
+
+
+def attn_jvp_fwd(q, k, v, tq, tk, tv, o, to, lse, B, H, Lq, Lk, D, scale, flags=0) -> int:
+    """Raw call: tensors (or integer device addresses) in, return code out.  See include/attn_jvp.h."""
+    return int(load().attn_jvp_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(tq), _ptr(tk), _ptr(tv), _ptr(o), _ptr(to),
+                                   _ptr(lse), B, H, Lq, Lk, D, float(scale), int(flags)))
+
+
+def attn_jvp_fwd_stream(q, k, v, tq, tk, tv, o, to, lse, B, H, Lq, Lk, D, scale, flags, cuda_stream) -> int:
+    return int(load().attn_jvp_fwd_stream(_ptr(q), _ptr(k), _ptr(v), _ptr(tq), _ptr(tk), _ptr(tv), _ptr(o),
+                                          _ptr(to), _ptr(lse), B, H, Lq, Lk, D, float(scale), int(flags),
+                                          _ptr(cuda_stream)))
+
+
+def _check(t, name, shape):
+    if not t.is_cuda or t.dtype != torch.bfloat16 or tuple(t.shape) != shape or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CUDA bf16 tensor of shape {shape}")
+
+
+def attention_jvp(q, k, v, tq=None, tk=None, tv=None, scale=None, fwd_only=False, out=None):
+    """O, tO, LSE of Algorithm 2 for [B][L][H][D] bf16 CUDA tensors, on torch's current stream.
+
+    ``tk is None and tv is None`` selects the tangent-free K/V path (cross-attention on a constant
+    context); ``fwd_only`` runs the plain forward (returns tO = None).  ``out`` may supply
+    preallocated (o, to, lse).  Returns (o, to, lse).
+    """
+    B, Lq, H, D = q.shape
+    Lk = k.shape[1]
+    _check(q, "q", (B, Lq, H, D)); _check(k, "k", (B, Lk, H, D)); _check(v, "v", (B, Lk, H, D))
+    flags = 0
+    if fwd_only:
+        flags |= FWD_ONLY
+        tq = tk = tv = None
+    else:
+        _check(tq, "tq", (B, Lq, H, D))
+        if tk is None and tv is None:
+            flags |= KV_TANGENT_FREE
+        else:
+            _check(tk, "tk", (B, Lk, H, D)); _check(tv, "tv", (B, Lk, H, D))
+    if scale is None:
+        scale = 1.0 / math.sqrt(D)
+    if out is None:
+        o = torch.empty_like(q)
+        to = None if fwd_only else torch.empty_like(q)
+        lse = torch.empty((B, H, Lq), dtype=torch.float32, device=q.device)
+    else:
+        o, to, lse = out
+    with torch.cuda.device(q.device):
+        stream = torch.cuda.current_stream().cuda_stream
+        rc = attn_jvp_fwd_stream(q, k, v, tq, tk, tv, o, to, lse, B, H, Lq, Lk, D, scale, flags, stream)
+    if rc != 0:
+        raise AttnJvpError(rc, attn_jvp_strerror(rc))
+    return o, to, lse
+
+
+def attention_jvp_host(q, k, v, tq=None, tk=None, tv=None, scale=None, fwd_only=False, device="cuda:0"):
+    """Host-to-host convenience: (pinned) CPU bf16 tensors in, CPU tensors out.
+
+    Copies the inputs to ``device``, runs :func:`attention_jvp`, copies O, tO, LSE back and
+    synchronises.  Returns (o, to, lse) on the CPU.
+    """
+    dev = torch.device(device)
+    up = lambda t: None if t is None else t.to(dev, non_blocking=True)
+    o, to, lse = attention_jvp(up(q), up(k), up(v), up(tq), up(tk), up(tv), scale=scale, fwd_only=fwd_only)
+    res = tuple(None if t is None else t.to("cpu", non_blocking=False) for t in (o, to, lse))
+    st = attn_jvp_device_status()
+    if st != 0:
+        raise AttnJvpError(st, attn_jvp_strerror(st))
+    return res

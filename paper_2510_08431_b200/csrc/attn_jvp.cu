@@ -1,0 +1,236 @@
+// Host side of the attention-JVP library: argument validation, TMA tensor maps, launch.
+// The C ABI is declared in include/attn_jvp.h.
+#include "attn_jvp.h"
+
+#include <cmath>
+#include <cstdint>
+#include <cstdio>
+#include <cstring>
+
+#include "attn_jvp_kernel.cuh"
+
+namespace {
+
+using attn_jvp::KernelArgs;
+
+constexpr int kVersion = 100;   // 0.1.0
+constexpr int kMaxDevices = 64;
+
+thread_local cudaStream_t tl_stream = nullptr;
+thread_local char tl_cuda_msg[256] = "";
+thread_local char tl_strerror_buf[384];
+
+int* g_host_status[kMaxDevices] = {};       // mapped pinned host words, one per device
+int* g_host_status_dev[kMaxDevices] = {};   // their device-side addresses
+bool g_smem_attr_set[kMaxDevices][2][3] = {};
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode_tiled = nullptr;
+
+int cuda_fail(const char* what, cudaError_t e) {
+    snprintf(tl_cuda_msg, sizeof tl_cuda_msg, "%s: %s", what, cudaGetErrorString(e));
+    return ATTN_JVP_ERR_CUDA;
+}
+
+int get_encode_fn() {
+    if (g_encode_tiled) return 0;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) return cuda_fail("cudaGetDriverEntryPoint(cuTensorMapEncodeTiled)", e);
+    if (qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+        snprintf(tl_cuda_msg, sizeof tl_cuda_msg, "cuTensorMapEncodeTiled not available from this driver");
+        return ATTN_JVP_ERR_CUDA;
+    }
+    g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    return 0;
+}
+
+// bf16 [B][L][H][D] tensor seen as a rank-4 map {D, H, L, B}; one box = 64 columns x `rows` rows
+// of one head, laid out in shared memory with the 128-byte swizzle the MMA descriptors expect.
+int make_map(CUtensorMap* map, const void* base, int B, int L, int H, int D, int rows) {
+    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)L, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)H * D * 2, (cuuint64_t)L * H * D * 2};
+    const cuuint32_t box[4] = {64, 1, (cuuint32_t)rows, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
+                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(tl_cuda_msg, sizeof tl_cuda_msg, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+        return ATTN_JVP_ERR_CUDA;
+    }
+    return 0;
+}
+
+bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+    if (!a || !b || na == 0 || nb == 0) return false;
+    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return a0 < b0 + nb && b0 < a0 + na;
+}
+
+template <int D, int MODE>
+int launch(const CUtensorMap* maps, const KernelArgs& ka, dim3 grid, cudaStream_t stream, int dev) {
+    auto kern = attn_jvp::attn_jvp_fwd_kernel<D, MODE>;
+    constexpr int smem = attn_jvp::SmemPlan<D>::kDynBytes;
+    bool& attr_set = g_smem_attr_set[dev][D == 128][MODE];
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
+        attr_set = true;
+    }
+    kern<<<grid, attn_jvp::kThreads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], ka);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail("kernel launch", e);
+    return 0;
+}
+
+int run(const void* q, const void* k, const void* v, const void* tq, const void* tk, const void* tv,
+        void* o, void* to, float* lse, int B, int H, int Lq, int Lk, int D, float scale, unsigned flags,
+        cudaStream_t stream) {
+    // ---- validation: nothing is enqueued unless everything checks out ----
+    if (flags & ~(ATTN_JVP_KV_TANGENT_FREE | ATTN_JVP_FWD_ONLY)) return ATTN_JVP_ERR_FLAGS;
+    const bool fwd_only = (flags & ATTN_JVP_FWD_ONLY) != 0;
+    const bool kv_free = (flags & ATTN_JVP_KV_TANGENT_FREE) != 0;
+    const int mode = fwd_only ? attn_jvp::kModeFwdOnly : (kv_free ? attn_jvp::kModeKvTangentFree : attn_jvp::kModeJvp);
+    if (B < 1 || H < 1 || Lq < 1 || Lk < 1) return ATTN_JVP_ERR_SHAPE;
+    if (D != 64 && D != 128) return ATTN_JVP_ERR_UNSUPPORTED_D;
+    if (B > 65535 || H > 65535) return ATTN_JVP_ERR_SHAPE;   // grid y / z limits
+    const long double nq = (long double)B * H * Lq * D, nk = (long double)B * H * Lk * D;
+    if (nq * 2 > 9.0e18L || nk * 2 > 9.0e18L) return ATTN_JVP_ERR_SHAPE;
+    if (!q || !k || !v || !o || !lse) return ATTN_JVP_ERR_NULL;
+    if (!fwd_only && (!tq || !to)) return ATTN_JVP_ERR_NULL;
+    if (mode == attn_jvp::kModeJvp && (!tk || !tv)) return ATTN_JVP_ERR_NULL;
+    if (!std::isfinite(scale)) return ATTN_JVP_ERR_SCALE;
+    const void* used_in[6] = {q, k, v, fwd_only ? nullptr : tq, mode == attn_jvp::kModeJvp ? tk : nullptr,
+                              mode == attn_jvp::kModeJvp ? tv : nullptr};
+    void* used_out[3] = {o, fwd_only ? nullptr : to, lse};
+    for (const void* p : used_in) if (p && ((uintptr_t)p & 15u)) return ATTN_JVP_ERR_ALIGN;
+    for (const void* p : used_out) if (p && ((uintptr_t)p & 15u)) return ATTN_JVP_ERR_ALIGN;
+    const size_t q_bytes = (size_t)B * Lq * H * D * 2, k_bytes = (size_t)B * Lk * H * D * 2;
+    const size_t lse_bytes = (size_t)B * H * Lq * 4;
+    const size_t in_bytes[6] = {q_bytes, k_bytes, k_bytes, q_bytes, k_bytes, k_bytes};
+    const size_t out_bytes[3] = {q_bytes, q_bytes, lse_bytes};
+    for (int a = 0; a < 3; ++a) {
+        for (int i = 0; i < 6; ++i)
+            if (overlaps(used_out[a], out_bytes[a], used_in[i], in_bytes[i])) return ATTN_JVP_ERR_ALIAS;
+        for (int c = a + 1; c < 3; ++c)
+            if (overlaps(used_out[a], out_bytes[a], used_out[c], out_bytes[c])) return ATTN_JVP_ERR_ALIAS;
+    }
+
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail("cudaGetDevice", e);
+    if (dev < 0 || dev >= kMaxDevices) return ATTN_JVP_ERR_ARCH;
+    int major = 0;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail("cudaDeviceGetAttribute", e);
+    if (major != 10) return ATTN_JVP_ERR_ARCH;
+
+    if (int rc = get_encode_fn()) return rc;
+    if (!g_host_status[dev]) {
+        int* hp = nullptr;
+        e = cudaHostAlloc((void**)&hp, sizeof(int), cudaHostAllocMapped);
+        if (e != cudaSuccess) return cuda_fail("cudaHostAlloc(status word)", e);
+        *hp = 0;
+        int* dp = nullptr;
+        e = cudaHostGetDevicePointer((void**)&dp, hp, 0);
+        if (e != cudaSuccess) { cudaFreeHost(hp); return cuda_fail("cudaHostGetDevicePointer", e); }
+        g_host_status[dev] = hp;
+        g_host_status_dev[dev] = dp;
+    }
+
+    // ---- tensor maps (Q-side boxes are 128 rows, K-side boxes 64 rows) ----
+    CUtensorMap maps[6];
+    if (int rc = make_map(&maps[0], q, B, Lq, H, D, attn_jvp::kBlockM)) return rc;
+    if (int rc = make_map(&maps[1], k, B, Lk, H, D, attn_jvp::kBlockN)) return rc;
+    if (int rc = make_map(&maps[2], v, B, Lk, H, D, attn_jvp::kBlockN)) return rc;
+    if (int rc = make_map(&maps[3], fwd_only ? q : tq, B, Lq, H, D, attn_jvp::kBlockM)) return rc;
+    if (int rc = make_map(&maps[4], mode == attn_jvp::kModeJvp ? tk : k, B, Lk, H, D, attn_jvp::kBlockN)) return rc;
+    if (int rc = make_map(&maps[5], mode == attn_jvp::kModeJvp ? tv : v, B, Lk, H, D, attn_jvp::kBlockN)) return rc;
+
+    KernelArgs ka;
+    ka.o = reinterpret_cast<__nv_bfloat16*>(o);
+    ka.to = reinterpret_cast<__nv_bfloat16*>(to);
+    ka.lse = lse;
+    ka.host_status = g_host_status_dev[dev];
+    ka.H = H;
+    ka.Lq = Lq;
+    ka.Lk = Lk;
+    ka.n_kv_tiles = (Lk + attn_jvp::kBlockN - 1) / attn_jvp::kBlockN;
+    ka.scale = scale;
+    ka.scale_log2 = scale * 1.4426950408889634f;
+
+    const dim3 grid((Lq + attn_jvp::kBlockM - 1) / attn_jvp::kBlockM, H, B);
+    if (D == 128) {
+        switch (mode) {
+            case attn_jvp::kModeJvp: return launch<128, attn_jvp::kModeJvp>(maps, ka, grid, stream, dev);
+            case attn_jvp::kModeKvTangentFree: return launch<128, attn_jvp::kModeKvTangentFree>(maps, ka, grid, stream, dev);
+            default: return launch<128, attn_jvp::kModeFwdOnly>(maps, ka, grid, stream, dev);
+        }
+    }
+    switch (mode) {
+        case attn_jvp::kModeJvp: return launch<64, attn_jvp::kModeJvp>(maps, ka, grid, stream, dev);
+        case attn_jvp::kModeKvTangentFree: return launch<64, attn_jvp::kModeKvTangentFree>(maps, ka, grid, stream, dev);
+        default: return launch<64, attn_jvp::kModeFwdOnly>(maps, ka, grid, stream, dev);
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+int attn_jvp_fwd(const void* q, const void* k, const void* v, const void* tq, const void* tk, const void* tv,
+                 void* o, void* to, float* lse, int B, int H, int Lq, int Lk, int D, float scale, unsigned flags) {
+    return run(q, k, v, tq, tk, tv, o, to, lse, B, H, Lq, Lk, D, scale, flags, tl_stream);
+}
+
+int attn_jvp_fwd_stream(const void* q, const void* k, const void* v, const void* tq, const void* tk, const void* tv,
+                        void* o, void* to, float* lse, int B, int H, int Lq, int Lk, int D, float scale,
+                        unsigned flags, void* cuda_stream) {
+    return run(q, k, v, tq, tk, tv, o, to, lse, B, H, Lq, Lk, D, scale, flags, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int attn_jvp_set_stream(void* cuda_stream) {
+    tl_stream = static_cast<cudaStream_t>(cuda_stream);
+    return 0;
+}
+
+int attn_jvp_device_status(void) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    int* hp = g_host_status[dev];
+    if (!hp) return 0;
+    const int st = *reinterpret_cast<volatile int*>(hp);
+    if (st != 0) {
+        *reinterpret_cast<volatile int*>(hp) = 0;
+        const int zero = 0;
+        cudaMemcpyToSymbol(attn_jvp::g_abort_flag, &zero, sizeof(int));   // let later launches run again
+    }
+    return st;
+}
+
+const char* attn_jvp_strerror(int code) {
+    switch (code) {
+        case ATTN_JVP_OK: return "ok";
+        case ATTN_JVP_ERR_NULL: return "a required pointer is NULL";
+        case ATTN_JVP_ERR_SHAPE: return "B, H, Lq and Lk must be >= 1 (B, H <= 65535) and sizes must not overflow";
+        case ATTN_JVP_ERR_UNSUPPORTED_D: return "head dimension D must be 64 or 128";
+        case ATTN_JVP_ERR_ALIGN: return "tensor pointers must be 16-byte aligned";
+        case ATTN_JVP_ERR_FLAGS: return "unknown flag bits";
+        case ATTN_JVP_ERR_SCALE: return "scale must be finite";
+        case ATTN_JVP_ERR_ALIAS: return "an output buffer overlaps an input or another output";
+        case ATTN_JVP_ERR_ARCH: return "the current device is not compute capability 10.x (sm_100a)";
+        case ATTN_JVP_ERR_CUDA:
+            snprintf(tl_strerror_buf, sizeof tl_strerror_buf, "CUDA call failed: %s", tl_cuda_msg);
+            return tl_strerror_buf;
+        case ATTN_JVP_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired; the kernel stopped early";
+        default: return "unknown error code";
+    }
+}
+
+int attn_jvp_version(void) { return kVersion; }
+
+}  // extern "C"
