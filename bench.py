@@ -1,0 +1,342 @@
+#!/usr/bin/env python
+"""Benchmark of the attention-JVP hot path (one step = one attn_jvp_fwd call over one synthetic batch).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is TFLOP/s counted as 12*B*H*Lq*Lk*D per call with the inputs
+resident in HBM; `e2e` is the same metric with pinned-host inputs copied in and O, tO, LSE copied out inside
+the timed region; `roofline` relates the kernel's average launch time (CUDA events on the launching stream)
+to the measured dense bf16 tensor peak; `cpu_baseline` times the fp64 oracle on the host cores on a bounded
+sample of the same workload.  With N > 1 every rank runs an independent replica (the path has no exchange
+step); the timed region is bracketed by a barrier and the time is the max over ranks.
+
+`--impl reference` times the fp64 oracle (there is no reference implementation to install: the paper
+ships no code), each step a bounded row sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from paper_2510_08431_b200 import synth  # noqa: E402
+
+METRIC = "attention-JVP TFLOP/s (12*B*H*Lq*Lk*D)"
+UNIT = "TFLOP/s"
+FALLBACK_BF16_TFLOPS = 1590.0   # earlier measurement on this machine, used only if MEASURED_PEAKS.json is absent
+DATASHEET_BF16_TFLOPS = 2250.0
+
+# DRAM bytes per launch of attn_jvp_fwd_kernel<128, jvp> measured with ncu (dram__bytes_read.sum +
+# dram__bytes_write.sum) on the image_dit_2b workload, see profiles/; scaled to other workloads by their
+# algorithmic bytes (traffic is proportional to the tensors streamed once from HBM; K/V re-reads hit L2).
+NCU_TRAFFIC_BYTES = {"workload": "image_dit_2b", "bytes": None}
+
+
+def algorithmic_bytes(w) -> int:
+    """Bytes that must cross HBM once: the six inputs, O, tO (bf16) and LSE (fp32)."""
+    q = w.B * w.Lq * w.H * w.D * 2
+    k = w.B * w.Lk * w.H * w.D * 2
+    n_in = 2 * q + (2 if w.kv_tangent_free else 4) * k
+    return n_in + 2 * q + w.B * w.H * w.Lq * 4
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"bf16_tflops": float(p["bf16_tflops"]), "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", 0)),
+                "source": "measured"}
+    return {"bf16_tflops": FALLBACK_BF16_TFLOPS, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); pw.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "power_w_max": max(pw),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def time_oracle(w, x_host, budget_s: float):
+    """Times the fp64 oracle (as it stands) on a row sample sized for about `budget_s` seconds."""
+    from oracle import attn_jvp_oracle as orc
+    orc.build()
+    bits = {k: (None if t is None else synth.bf16_bits(t)) for k, t in x_host.items()}
+    n_total = w.B * w.H * w.Lq
+    per_row = (8 if w.kv_tangent_free else 12) * w.Lk * w.D
+
+    def run(n):
+        # rows of one head, spread over the sequence (one head => one K/V widening, like a real call per head)
+        rows = np.unique(np.linspace(0, w.Lq - 1, num=min(n, w.Lq)).astype(np.int64))
+        t0 = time.perf_counter()
+        orc.attn_jvp_def_bf16_rows(bits["q"], bits["k"], bits["v"], bits["tq"], bits["tk"], bits["tv"],
+                                   w.B, w.H, w.Lq, w.Lk, w.D, w.scale, rows)
+        return len(rows), time.perf_counter() - t0
+
+    n0, t_probe = run(64)
+    rate = n0 / max(t_probe, 1e-6)
+    n = int(max(64, min(n_total, w.Lq, rate * budget_s)))
+    n, dt = run(n)
+    nominal_per_row = 12 * w.Lk * w.D
+    return {"value": n * nominal_per_row / dt / 1e12, "unit": UNIT, "cores": orc.threads(), "kind": "oracle",
+            "sample": f"{n} query rows of head (b=0,h=0) against all {w.Lk} keys, fp64, {dt:.1f} s "
+                      f"({n / dt:.1f} rows/s; executed {per_row} flop/row, counted {nominal_per_row})",
+            "seconds": dt, "rows": n}
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    x = synth.make_workload(w)
+    times, rows = [], 0
+    budget = max(2.0, min(20.0, 120.0 / max(1, args.steps + args.warmup)))
+    res = None
+    for i in range(args.warmup + args.steps):
+        res = time_oracle(w, x, budget)
+        if i >= args.warmup:
+            times.append(res["seconds"]); rows += res["rows"]
+    total = sum(times)
+    value = rows * 12 * w.Lk * w.D / total / 1e12
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(w, extra={"reference": "fp64 CPU oracle; each step a bounded row sample"}),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": res["cores"], "kind": "oracle",
+                             "sample": res["sample"]},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w, extra=None):
+    cfg = {"workload": w.name, "B": w.B, "H": w.H, "Lq": w.Lq, "Lk": w.Lk, "D": w.D, "scale": w.scale,
+           "kv_tangent_free": w.kv_tangent_free, "layout": "BLHD bf16", "seed": w.seed,
+           "parallelism": "replicas only (no collective on the path)",
+           "l2": "inputs larger than L2 (no flush needed)" if algorithmic_bytes(w) > 2 * 126e6 else "L2 flushed between timed iterations"}
+    if extra:
+        cfg.update(extra)
+    return cfg
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="video_dit_14b", choices=sorted(synth.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    w = synth.WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import paper_2510_08431_b200 as aj
+    aj.load()   # raises if the CUDA library is missing: there is no fallback
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (sm_100a); there is no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # each rank draws its own replica of the workload (seed offset by rank)
+    x_host = synth.make_inputs(w.B, w.H, w.Lq, w.Lk, w.D, w.sigma_primal, w.sigma_tangent, w.seed + 1000 * rank,
+                               w.kv_tangent_free, pin_memory=not args.no_e2e)
+    g = {k: (None if t is None else t.to(dev)) for k, t in x_host.items()}
+    o = torch.empty_like(g["q"]); to = torch.empty_like(g["q"])
+    lse = torch.empty((w.B, w.H, w.Lq), dtype=torch.float32, device=dev)
+    flush = None
+    if algorithmic_bytes(w) <= 2 * 126e6:
+        flush = torch.empty(512 * 1024 * 1024, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(fwd_only=False):
+        aj.attention_jvp(g["q"], g["k"], g["v"], g["tq"], g["tk"], g["tv"], scale=w.scale, fwd_only=fwd_only,
+                         out=(o, None if fwd_only else to, lse))
+
+    def timed(n_steps, fwd_only=False):
+        """Per-launch CUDA-event durations (ms) on the launching stream."""
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_steps)]
+        for a, b in evs:
+            if flush is not None:
+                flush.zero_()
+            a.record(stream)
+            step(fwd_only)
+            b.record(stream)
+        torch.cuda.synchronize()
+        return [a.elapsed_time(b) for a, b in evs]
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    st = aj.attn_jvp_device_status()
+    if st != 0:
+        raise RuntimeError(aj.attn_jvp_strerror(st))
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    t_begin = torch.cuda.Event(enable_timing=True); t_end = torch.cuda.Event(enable_timing=True)
+    t_begin.record(stream)
+    per_launch = timed(args.steps)
+    t_end.record(stream)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    kernel_ms = sum(per_launch) / len(per_launch)
+    total_ms = t_begin.elapsed_time(t_end) if flush is None else sum(per_launch)
+    tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    value = world * w.flops / (ms_per_step * 1e-3) / 1e12
+
+    # forward-only of the same kernel, for the JVP / forward cost ratio
+    fwd_ms = None
+    if not w.kv_tangent_free:
+        timed(2, fwd_only=True)
+        f = timed(max(3, args.steps // 2), fwd_only=True)
+        fwd_ms = sum(f) / len(f)
+
+    # end to end: pinned host inputs -> device, kernel, O / tO / LSE -> pinned host, every step
+    e2e = None
+    if not args.no_e2e:
+        ho = torch.empty(o.shape, dtype=o.dtype, pin_memory=True)
+        hto = torch.empty(o.shape, dtype=o.dtype, pin_memory=True)
+        hl = torch.empty(lse.shape, dtype=lse.dtype, pin_memory=True)
+        names = [k for k in ("q", "k", "v", "tq", "tk", "tv") if x_host[k] is not None]
+        h2d = sum(x_host[k].numel() * 2 for k in names)
+        d2h = ho.numel() * 2 + hto.numel() * 2 + hl.numel() * 4
+
+        def e2e_step():
+            for k in names:
+                g[k].copy_(x_host[k], non_blocking=True)
+            step()
+            ho.copy_(o, non_blocking=True); hto.copy_(to, non_blocking=True); hl.copy_(lse, non_blocking=True)
+
+        e2e_step(); torch.cuda.synchronize()
+        barrier()
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        n_e2e = max(2, min(args.steps, 5))
+        a.record(stream)
+        for _ in range(n_e2e):
+            e2e_step()
+        b.record(stream)
+        barrier()
+        et = torch.tensor([a.elapsed_time(b)], dtype=torch.float64, device=dev)
+        if dist is not None:
+            dist.all_reduce(et, op=dist.ReduceOp.MAX)
+        e2e_ms = float(et.item()) / n_e2e
+        e2e = {"value": world * w.flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": n_e2e}
+    st = aj.attn_jvp_device_status()
+    if st != 0:
+        raise RuntimeError(aj.attn_jvp_strerror(st))
+
+    if rank == 0:
+        peaks = measured_peaks()
+        flops = w.executed_flops
+        achieved = flops / (kernel_ms * 1e-3) / 1e12
+        traffic = None
+        if NCU_TRAFFIC_BYTES["bytes"] is not None:
+            wt = synth.WORKLOADS[NCU_TRAFFIC_BYTES["workload"]]
+            traffic = NCU_TRAFFIC_BYTES["bytes"] * algorithmic_bytes(w) / algorithmic_bytes(wt)
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                    "frac": achieved / peaks["bf16_tflops"], "traffic": traffic,
+                    "peak_source": f"{peaks['source']} burst cuBLAS bf16 (MEASURED_PEAKS.json)",
+                    "kernel": "attn_jvp_fwd_kernel", "kernel_ms": kernel_ms, "flops_per_launch": flops,
+                    "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None,
+                    "frac_of_datasheet": achieved / DATASHEET_BF16_TFLOPS,
+                    "algorithmic_bytes": algorithmic_bytes(w)}
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": workload_config(w), "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps,
+                "roofline": roofline,
+                "jvp_over_fwd": (kernel_ms / fwd_ms) if fwd_ms else None, "fwd_only_ms": fwd_ms,
+                "per_launch_ms": {"median": statistics.median(per_launch), "best": min(per_launch)}}
+        if world == 1 and not args.no_cpu_baseline:
+            cb = time_oracle(w, x_host, 15.0)
+            line["cpu_baseline"] = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

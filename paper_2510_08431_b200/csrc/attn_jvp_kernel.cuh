@@ -456,7 +456,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const bool neg_scale = c1 < 0.0f;
         float m_ref = -INFINITY;   // running reference max, log2 domain (m of Algorithm 2, lazily updated)
         float l_run = 0.0f;        // l
-        float r_run = 0.0f;        // r
+        float r_run = 0.0f;        // r (of the centred tS, see below)
+        float ts_shift = 0.0f;     // per-row constant subtracted from tS
         bool ok = true;
 
         for (int j = 0; j < n_kv; ++j) {
@@ -546,11 +547,21 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 TMEM_ST32(tm_s, pk, 0);
             }
             if (kHasTQ) {
+                // tO does not change when a per-row constant is subtracted from tS (softmax is shift
+                // invariant: the constant leaves H~ V - (r/l) O unchanged).  Centring tS on its P-weighted
+                // mean over the first tile keeps H~ and r small, so that the bf16 rounding of H~ scales
+                // with |tS - mu| instead of |tS| when the two terms cancel in the epilogue.
+                if (j == 0) {
+                    float num = 0.0f;
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) num = fmaf(__uint_as_float(sv[c]), __uint_as_float(tv[c]) * sc, num);
+                    ts_shift = num / lsum;
+                }
                 // H~ = P~ . tS, r += rowsum(H~)
                 float rsum = 0.0f;
 #pragma unroll
                 for (int c = 0; c < 64; ++c) {
-                    const float hv = __uint_as_float(sv[c]) * (__uint_as_float(tv[c]) * sc);
+                    const float hv = __uint_as_float(sv[c]) * fmaf(__uint_as_float(tv[c]), sc, -ts_shift);
                     tv[c] = __float_as_uint(hv);
                     rsum += hv;
                 }

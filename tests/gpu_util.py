@@ -1,0 +1,59 @@
+"""Helpers of the GPU parity tests (test harness only)."""
+import numpy as np
+import torch
+
+from paper_2510_08431_b200 import synth
+
+TOL = 2e-2          # max |err| <= TOL * (1 + |ref|) on O and tO: bf16 in, fp32 accumulate
+REL_L2 = 1e-2       # supplementary: ||gpu - ref||_2 / ||ref||_2 (the max-norm gate is loose at long Lk)
+LSE_TOL = 1e-3      # |err| <= LSE_TOL * (1 + |ref|)
+
+
+def to_gpu(x):
+    return {k: (None if t is None else t.cuda()) for k, t in x.items()}
+
+
+def rows_of(t, rows, D):
+    """[B][L][H][D] tensor -> fp64 numpy [n][D] for flat rows (b*H + h)*L + i."""
+    B, L, H, _ = t.shape
+    idx = torch.as_tensor(np.asarray(rows), dtype=torch.long)
+    bh, i = idx // L, idx % L
+    b, h = bh // H, bh % H
+    return t.cpu()[b, i, h, :].double().numpy()
+
+
+def oracle_rows(oracle, x, B, H, Lq, Lk, D, scale, rows):
+    bits = {k: (None if t is None else synth.bf16_bits(t)) for k, t in x.items()}
+    return oracle.attn_jvp_def_bf16_rows(bits["q"], bits["k"], bits["v"], bits["tq"], bits["tk"], bits["tv"],
+                                         B, H, Lq, Lk, D, scale, rows)
+
+
+def check(name, got, ref, tol=TOL, rel=REL_L2, cancel=None):
+    """The mandated max-norm gate plus a relative-L2 gate.  For tO, `cancel` = mu * O (fp64, from the
+    oracle): tO is the difference of the accumulated H~ V term and mu * O, so its rounding error scales
+    with those terms, not with tO itself (with one key and tK = tV = 0 the exact tO is 0)."""
+    assert np.isfinite(got).all(), f"{name}: non-finite values"
+    ratio = np.abs(got - ref) / (tol * (1 + np.abs(ref)))
+    assert ratio.max() <= 1.0, f"{name}: max err/tol = {ratio.max():.3g}"
+    if rel is not None:
+        denom = np.linalg.norm(ref) + (np.linalg.norm(cancel) if cancel is not None else 0.0)
+        r = np.linalg.norm(got - ref) / max(denom, 1e-30)
+        assert r <= rel, f"{name}: rel-L2 = {r:.3g}"
+
+
+def check_all(oracle, aj, x, B, H, Lq, Lk, D, scale, rows, o, to, lse, rel=REL_L2):
+    rO, rtO, rL, rMU = oracle_rows(oracle, x, B, H, Lq, Lk, D, scale, rows)
+    check("O", rows_of(o, rows, D), rO, rel=rel)
+    if to is not None:
+        check("tO", rows_of(to, rows, D), rtO, rel=rel, cancel=rMU[:, None] * rO)
+    gL = lse.cpu().reshape(-1).double().numpy()[np.asarray(rows)]
+    assert (np.abs(gL - rL) <= LSE_TOL * (1 + np.abs(rL))).all(), f"LSE: max err {np.abs(gL - rL).max():.3g}"
+
+
+def run(aj, g, scale, fwd_only=False, out=None):
+    o, to, lse = aj.attention_jvp(g["q"], g["k"], g["v"], g["tq"], g["tk"], g["tv"], scale=scale,
+                                  fwd_only=fwd_only, out=out)
+    torch.cuda.synchronize()
+    st = aj.attn_jvp_device_status()
+    assert st == 0, aj.attn_jvp_strerror(st)
+    return o, to, lse

@@ -1,0 +1,76 @@
+"""The five benchmark workloads at full size, in the launch configuration the benchmark times:
+sampled query rows against the fp64 oracle (each sampled row against ALL keys), plus whole-tensor
+coverage through a chunked fp32 comparator that is itself checked against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2510_08431_b200 import synth
+from tests import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def aj():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    from paper_2510_08431_b200 import build
+    build.build_library()
+    import paper_2510_08431_b200 as aj
+    aj.load()
+    return aj
+
+
+def _fp32_comparator(g, scale, b, h, rows):
+    """Plain fp32 attention JVP for query rows `rows` of one head on the GPU (test harness only)."""
+    torch.backends.cuda.matmul.allow_tf32 = False
+    f = lambda t: None if t is None else t[b, :, h, :].float()
+    q, tq = f(g["q"])[rows], f(g["tq"])[rows]
+    k, v, tk, tv = f(g["k"]), f(g["v"]), f(g["tk"]), f(g["tv"])
+    s = scale * q @ k.T
+    ts = scale * (tq @ k.T)
+    if tk is not None:
+        ts = ts + scale * (q @ tk.T)
+    p = torch.softmax(s, dim=-1)
+    mu = (p * ts).sum(-1, keepdim=True)
+    o = p @ v
+    to = (p * (ts - mu)) @ v
+    if tv is not None:
+        to = to + p @ tv
+    return o, to, torch.logsumexp(s, dim=-1)
+
+
+@pytest.mark.parametrize("name,n_rand,full_tiles,heads_full", [
+    ("image_dit_2b", 8, (0, 17), (0, 31)),
+    ("video_dit_1p3b", 3, (0,), (0,)),
+    ("video_dit_14b", 2, (0, 127), (0, 39)),
+    ("cross_attn_14b", 8, (0, 100), (0, 39)),
+])
+def test_full_size_workload(aj, oracle, name, n_rand, full_tiles, heads_full):
+    w = synth.WORKLOADS[name]
+    x = synth.make_workload(w)
+    g = U.to_gpu(x)
+    o, to, lse = U.run(aj, g, w.scale)
+    rows = synth.sample_rows(w.B, w.H, w.Lq, n_random_per_head=n_rand, tile=128, full_tiles=full_tiles,
+                             heads_full=heads_full, seed=w.seed)
+    U.check_all(oracle, aj, x, w.B, w.H, w.Lq, w.Lk, w.D, w.scale, rows, o, to, lse)
+
+    # whole-tensor coverage for a few heads: fp32 comparator (pinned to the oracle on sampled rows)
+    rO, rtO, rL, _ = U.oracle_rows(oracle, x, w.B, w.H, w.Lq, w.Lk, w.D, w.scale, rows[:64])
+    for n, r in enumerate(rows[:64]):
+        bh, i = divmod(r, w.Lq)
+        co, cto, cl = _fp32_comparator(g, w.scale, bh // w.H, bh % w.H, torch.tensor([i], device="cuda"))
+        assert np.abs(co[0].double().cpu().numpy() - rO[n]).max() <= 1e-4
+        assert np.abs(cto[0].double().cpu().numpy() - rtO[n]).max() <= 1e-4
+    heads = [(0, 0), (w.B - 1, w.H - 1)]
+    chunk = 2048
+    for b, h in heads:
+        worst_o = worst_t = 0.0
+        for r0 in range(0, w.Lq, chunk):
+            rr = torch.arange(r0, min(w.Lq, r0 + chunk), device="cuda")
+            co, cto, cl = _fp32_comparator(g, w.scale, b, h, rr)
+            eo = (o[b, rr, h, :].float() - co).abs() / (U.TOL * (1 + co.abs()))
+            et = (to[b, rr, h, :].float() - cto).abs() / (U.TOL * (1 + cto.abs()))
+            worst_o, worst_t = max(worst_o, eo.max().item()), max(worst_t, et.max().item())
+            assert (lse[b, h, rr] - cl).abs().max().item() <= 1e-3 * (1 + cl.abs().max().item())
+        assert worst_o <= 1.0 and worst_t <= 1.0, (worst_o, worst_t)
