@@ -59,6 +59,7 @@ extern "C" {
 #define ATTN_JVP_ERR_ARCH            8  /* current device is not compute capability 10.x */
 #define ATTN_JVP_ERR_CUDA            9  /* a CUDA runtime / driver call failed (see strerror) */
 #define ATTN_JVP_ERR_DEVICE_TIMEOUT 10  /* a bounded device-side wait expired */
+#define ATTN_JVP_ERR_DEVICE_LAYOUT  11  /* the kernel's shared-memory layout did not fit (reported like a timeout) */
 
 /*
  * attn_jvp_fwd -- O, tO and LSE of Algorithm 2 in one pass, on the stream set
@@ -91,8 +92,9 @@ int attn_jvp_set_stream(void* cuda_stream);
 /*
  * Device-side status of the current device since the last call of this
  * function: 0, or ATTN_JVP_ERR_DEVICE_TIMEOUT if a bounded wait inside a
- * kernel expired.  Meaningful once the caller has synchronised the stream(s)
- * the kernels ran on; reading it clears it.  Does not synchronise.
+ * kernel expired (ATTN_JVP_ERR_DEVICE_LAYOUT if its shared-memory layout did
+ * not fit).  Meaningful once the caller has synchronised the stream(s) the
+ * kernels ran on; reading it clears it.  Does not synchronise.
  */
 int attn_jvp_device_status(void);
 

@@ -17,7 +17,7 @@ KV_TANGENT_FREE = 0x1
 FWD_ONLY = 0x2
 
 ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED_D, ERR_ALIGN, ERR_FLAGS = 1, 2, 3, 4, 5
-ERR_SCALE, ERR_ALIAS, ERR_ARCH, ERR_CUDA, ERR_DEVICE_TIMEOUT = 6, 7, 8, 9, 10
+ERR_SCALE, ERR_ALIAS, ERR_ARCH, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_DEVICE_LAYOUT = 6, 7, 8, 9, 10, 11
 
 EXPORTS = ("attn_jvp_fwd", "attn_jvp_fwd_stream", "attn_jvp_set_stream", "attn_jvp_device_status",
            "attn_jvp_strerror", "attn_jvp_version")

@@ -22,7 +22,7 @@ thread_local char tl_strerror_buf[384];
 
 int* g_host_status[kMaxDevices] = {};       // mapped pinned host words, one per device
 int* g_host_status_dev[kMaxDevices] = {};   // their device-side addresses
-bool g_smem_attr_set[kMaxDevices][2][3] = {};
+int g_dyn_smem[kMaxDevices][2][3] = {};     // dynamic shared memory per kernel instantiation, 0 = not set up
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -74,12 +74,27 @@ bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
 template <int D, int MODE>
 int launch(const CUtensorMap* maps, const KernelArgs& ka, dim3 grid, cudaStream_t stream, int dev) {
     auto kern = attn_jvp::attn_jvp_fwd_kernel<D, MODE>;
-    constexpr int smem = attn_jvp::SmemPlan<D>::kDynBytes;
-    bool& attr_set = g_smem_attr_set[dev][D == 128][MODE];
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    int& smem = g_dyn_smem[dev][D == 128][MODE];
+    if (smem == 0) {
+        // dynamic shared memory = the operand layout plus slack for its 1024-byte alignment, capped by
+        // what the device leaves after the kernel's static shared memory
+        cudaFuncAttributes fa;
+        cudaError_t e = cudaFuncGetAttributes(&fa, kern);
+        if (e != cudaSuccess) return cuda_fail("cudaFuncGetAttributes", e);
+        int optin = 0;
+        e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+        if (e != cudaSuccess) return cuda_fail("cudaDeviceGetAttribute(MaxSharedMemoryPerBlockOptin)", e);
+        int want = attn_jvp::SmemPlan<D>::kDynBytes;
+        const int room = optin - (int)fa.sharedSizeBytes;
+        if (want > room) want = room;
+        if (want < attn_jvp::SmemPlan<D>::kBytes) {
+            snprintf(tl_cuda_msg, sizeof tl_cuda_msg, "device offers %d bytes of shared memory, kernel needs %d",
+                     room, attn_jvp::SmemPlan<D>::kBytes);
+            return ATTN_JVP_ERR_CUDA;
+        }
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, want);
         if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
-        attr_set = true;
+        smem = want;
     }
     kern<<<grid, attn_jvp::kThreads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], ka);
     cudaError_t e = cudaGetLastError();
@@ -227,10 +242,21 @@ const char* attn_jvp_strerror(int code) {
             snprintf(tl_strerror_buf, sizeof tl_strerror_buf, "CUDA call failed: %s", tl_cuda_msg);
             return tl_strerror_buf;
         case ATTN_JVP_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired; the kernel stopped early";
+        case ATTN_JVP_ERR_DEVICE_LAYOUT: return "the kernel's shared-memory layout did not fit; nothing was computed";
         default: return "unknown error code";
     }
 }
 
 int attn_jvp_version(void) { return kVersion; }
+
+#ifdef ATTN_JVP_TRACE
+// Debug builds only: copies the in-kernel timeline (clock64 stamps) of the traced CTA to `dst`.
+int attn_jvp_debug_read_trace(long long* dst, int n) {
+    const int total = attn_jvp::kTraceEvents * attn_jvp::kTraceSteps;
+    if (n < total) return -total;
+    cudaError_t e = cudaMemcpyFromSymbol(dst, attn_jvp::g_trace, sizeof(long long) * total);
+    return e == cudaSuccess ? total : -1;
+}
+#endif
 
 }  // extern "C"
