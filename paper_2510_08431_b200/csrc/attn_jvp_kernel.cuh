@@ -56,7 +56,11 @@ enum Mode : int { kModeJvp = 0, kModeKvTangentFree = 1, kModeFwdOnly = 2 };
 constexpr int kTraceSteps = 96;
 constexpr int kTraceEvents = 24;
 __device__ long long g_trace[kTraceEvents][kTraceSteps];
+#if ATTN_JVP_TRACE >= 2
 #define TRACE(evt, idx) do { if (trace_on && (idx) < kTraceSteps) g_trace[evt][idx] = clock64(); } while (0)
+#else
+#define TRACE(evt, idx) do { } while (0)     // level 1: only the CTA's begin / end stamps
+#endif
 #else
 #define TRACE(evt, idx) do { } while (0)
 #endif
@@ -328,6 +332,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     __syncthreads();
     if (cta_abort != 0) return;
 
+#ifdef ATTN_JVP_TRACE
+    if (trace_on && threadIdx.x == 0) g_trace[kTraceEvents - 1][0] = clock64();      // CTA begins
+#endif
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t smem_q = smem_base;
     const uint32_t smem_tq = smem_base + Plan::kQBytes;
@@ -484,11 +491,11 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 return mbar_wait_warp(bar, r.parity, abort_state);
             };
 
-            // score MMAs of tile j out of ring slot `slot` (issued by the elected lane)
-            auto issue_scores = [&](int j, int slot) {
+            // score MMAs of tile j out of ring slot `slot` (issued by the elected lane), in two parts so that
+            // the look-ahead for the next tile can run between them
+            auto issue_scores_a = [&](int j, int slot) {
                 const uint32_t k_lo = make_desc_lo(smem_ring + slot * Plan::kSlotBytes, 16);
                 const uint32_t tm_s = tmem + kScoreCol0 + (j & 1) * kScoreBufStride;
-                const uint32_t tm_ts = tm_s + kBlockN;
                 TRACE(21, j);         // MMA: about to issue score MMAs
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
@@ -496,6 +503,10 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const uint32_t boff = ((k / 4) * 2 * Plan::kKvHalfBytes + (k % 4) * 32) >> 4;
                     mma_ss(tm_s, q_lo + koff, k_lo + boff, kIdescS1, k > 0);
                 }
+            };
+            auto issue_scores_b = [&](int j, int slot) {
+                const uint32_t k_lo = make_desc_lo(smem_ring + slot * Plan::kSlotBytes, 16);
+                const uint32_t tm_ts = tmem + kScoreCol0 + (j & 1) * kScoreBufStride + kBlockN;
                 if (kHasTQ) {
 #pragma unroll
                     for (int k = 0; k < D / 16; ++k) {
@@ -528,43 +539,73 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 tc_commit(smem_u32(&bar_pv_done));
                 TRACE(4, j);          // MMA: value MMAs of tile j issued
             };
+            // what tile j's burst needs: V(j) and K(j+2) in shared memory, P~/H~ of tile j in tensor memory
+            auto test_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, int j) -> bool {
+                bool r = mbar_test_wait(smem_u32(&bar_slot_full[pv.slot]), pv.parity);
+                if (has_k) r = r && mbar_test_wait(smem_u32(&bar_slot_full[pk.slot]), pk.parity);
+                r = r && mbar_test_wait(smem_u32(&bar_p_full[j & 1]), (j >> 1) & 1);
+                return __all_sync(0xffffffffu, r);
+            };
+            auto wait_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, int j) -> bool {
+                if (leader) TRACE(22, j);   // MMA: has to block for tile j
+                bool r = wait_full(pv);
+                if (r && has_k) r = wait_full(pk);
+                if (r) r = mbar_wait_warp(smem_u32(&bar_p_full[j & 1]), (j >> 1) & 1, abort_state);
+                return r;
+            };
 
             // Ring order (as the producer fills it): K0, K1, V0, K2, V1, K3, ...
             RingPos pos{0, 0u};
             if (ok) ok = wait_full(pos);
             if (ok) {
                 tc_fence_after();
-                if (leader) issue_scores(0, pos.slot);
+                if (leader) { issue_scores_a(0, pos.slot); issue_scores_b(0, pos.slot); }
                 __syncwarp();
                 advance(pos);
             }
             if (ok && n_kv > 1) {
                 ok = wait_full(pos);
                 if (ok) {
-                    if (leader) issue_scores(1, pos.slot);
+                    if (leader) { issue_scores_a(1, pos.slot); issue_scores_b(1, pos.slot); }
                     __syncwarp();
                     advance(pos);
                 }
             }
-            for (int j = 0; ok && j < n_kv; ++j) {
-                const RingPos pos_v = pos;
+            // pos = V(0).  Per tile j: burst = value MMAs of tile j, score MMAs of tile j+2; the barriers of tile
+            // j+1 are tested in the middle of the burst, while the queue is still full.
+            RingPos pos_v = pos, pos_k = pos;
+            bool has_k = n_kv > 2;
+            if (ok) {
                 advance(pos);
-                const bool more = j + 2 < n_kv;
-                const RingPos pos_k = pos;
-                if (more) advance(pos);
-                if (leader) TRACE(22, j);
-                ok = wait_full(pos_v);                                   // V(j): almost always there already
-                if (ok && more) ok = wait_full(pos_k);                   // K(j+2): likewise
-                if (leader) TRACE(23, j);
-                if (ok) ok = mbar_wait_warp(smem_u32(&bar_p_full[j & 1]), (j >> 1) & 1, abort_state);
-                if (!ok) break;
-                if (leader) TRACE(1, j);
+                pos_k = pos;
+                if (has_k) advance(pos);
+                ok = wait_tile(pos_v, pos_k, has_k, 0);
+            }
+            for (int j = 0; ok && j < n_kv; ++j) {
+                // ring positions of the next tile
+                const RingPos nxt_v = pos;
+                RingPos nxt_k = pos;
+                const bool nxt_exists = j + 1 < n_kv;
+                const bool nxt_has_k = j + 3 < n_kv;
+                if (nxt_exists) {
+                    advance(pos);
+                    nxt_k = pos;
+                    if (nxt_has_k) advance(pos);
+                }
                 tc_fence_after();
                 if (leader) {
                     issue_values(j, pos_v.slot);
-                    if (more) issue_scores(j + 2, pos_k.slot);
+                    if (has_k) issue_scores_a(j + 2, pos_k.slot);
                 }
                 __syncwarp();
+                bool nxt_ready = true;
+                if (nxt_exists) nxt_ready = test_tile(nxt_v, nxt_k, nxt_has_k, j + 1);
+                if (leader && has_k) issue_scores_b(j + 2, pos_k.slot);
+                __syncwarp();
+                if (nxt_exists && !nxt_ready) ok = wait_tile(nxt_v, nxt_k, nxt_has_k, j + 1);
+                pos_v = nxt_v;
+                pos_k = nxt_k;
+                has_k = nxt_has_k;
             }
             if (!ok && leader) {
                 // Abandoning the tile: wait (bounded) until the tensor core has drained what was issued.
@@ -595,16 +636,12 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const int bsel = j & 1;
             if (!mbar_wait_warp(smem_u32(&bar_s_full[bsel]), (j >> 1) & 1, abort_state)) { ok = false; break; }
             tc_fence_after();
-#ifdef ATTN_JVP_TRACE
+#if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
             const bool trace_me = trace_on && lane == 0;
             if (trace_me && j < kTraceSteps) g_trace[5 + (warp - kFirstSoftmaxWarp)][j] = clock64();     // softmax warp: scores seen ready
 #endif
             const uint32_t tm_s = tmem + lane_base + kScoreCol0 + bsel * kScoreBufStride;
             const uint32_t tm_ts = tm_s + kBlockN;
-#ifdef ATTN_JVP_DEBUG_SKIP_SOFTMAX
-            // timing experiment only (wrong results): hand the tile straight back to the MMA warp
-            if (j >= 0) { l_run = 1.0f; tc_fence_before(); mbar_arrive(smem_u32(&bar_p_full[bsel])); continue; }
-#endif
 
             uint32_t sv[kHalfN];
             uint32_t tv[kHalfN];
@@ -735,7 +772,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             tc_wait_st();
             tc_fence_before();
             mbar_arrive(smem_u32(&bar_p_full[bsel]));
-#ifdef ATTN_JVP_TRACE
+#if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
             if (trace_me && j < kTraceSteps) g_trace[13 + (warp - kFirstSoftmaxWarp)][j] = clock64();    // softmax warp: arrived
 #endif
         }
@@ -807,6 +844,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // Teardown: every role falls through to here (all waits are bounded).
     tc_fence_before();
     __syncthreads();
+#ifdef ATTN_JVP_TRACE
+    if (trace_on && threadIdx.x == 0) g_trace[kTraceEvents - 1][1] = clock64();      // CTA ends
+#endif
     if (warp == kMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
