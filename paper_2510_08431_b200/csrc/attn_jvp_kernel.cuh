@@ -225,23 +225,32 @@ __device__ __forceinline__ uint32_t make_desc_lo(uint32_t addr, uint32_t lbo_byt
     return ((addr & 0x3FFFFu) >> 4) | ((lbo_bytes >> 4) << 16);
 }
 
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-        "mov.b64 da, {%1, %5};\n\tmov.b64 db, {%2, %5};\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi) : "memory");
+// Full 64-bit descriptor from its low word.
+__device__ __forceinline__ uint64_t make_desc(uint32_t lo) {
+    uint64_t d;
+    asm volatile("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(kDescHi));
+    return d;
 }
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
+// D[tmem] (+)= A[smem] * B[smem]; the accumulate flag is a compile-time choice so that nothing but the
+// MMA itself has to be issued per instruction.
+template <bool kAccumulate>
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+    if (kAccumulate) {
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.u32 p, 1, 1;\n\t"
+                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc) : "memory");
+    } else {
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, 1, 1;\n\t"
+                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc) : "memory");
+    }
+}
+// D[tmem] (+)= A[tmem] * B[smem]; runtime accumulate flag (the first value MMA of a query tile overwrites)
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
-        "mov.b64 db, {%2, %5};\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(kDescHi) : "memory");
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
 // 32 lanes x 32 columns: thread t of the warp receives columns [addr.col, +32) of lane (warp%4)*32 + t
@@ -282,6 +291,31 @@ __device__ __forceinline__ float ex2f(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// Two fp32 lanes per instruction (sm_100 packed fp32 arithmetic): halves the FMA-pipe instruction count
+// of the softmax inner loops.
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul_f32x2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&h);
@@ -310,7 +344,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     __shared__ __align__(8) uint64_t bar_p_full[2];
     __shared__ __align__(8) uint64_t bar_pv_done;
     __shared__ __align__(8) uint64_t bar_drain;
-    __shared__ __align__(8) uint64_t bar_xchg[3];   // [0],[1]: row maxima of even / odd tiles; [2]: partial sums
+    // Exchanges between the two warps that own the same 32 rows (quarter q = warp % 4): [0][q], [1][q] row
+    // maxima of even / odd key tiles, [2][q] partial sums.  One elected lane per warp arrives.
+    __shared__ __align__(8) uint64_t bar_xchg[3][4];
     __shared__ uint32_t tmem_base_smem;
     __shared__ int cta_abort;
     __shared__ float xchg_max[2][2][kBlockM];     // [tile parity][column half][row]: per-half row maxima
@@ -361,13 +397,12 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&bar_s_full[i]), 1);
-            mbar_init(smem_u32(&bar_p_full[i]), kSoftmaxThreads);
+            mbar_init(smem_u32(&bar_p_full[i]), kSoftmaxThreads / 32);    // one arrival per softmax warp
         }
         mbar_init(smem_u32(&bar_pv_done), 1);
         mbar_init(smem_u32(&bar_drain), 1);
-        mbar_init(smem_u32(&bar_xchg[0]), kSoftmaxThreads);
-        mbar_init(smem_u32(&bar_xchg[1]), kSoftmaxThreads);
-        mbar_init(smem_u32(&bar_xchg[2]), kSoftmaxThreads);
+        for (int i = 0; i < 3; ++i)
+            for (int q = 0; q < 4; ++q) mbar_init(smem_u32(&bar_xchg[i][q]), 2);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kMmaWarp) {
@@ -491,29 +526,47 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 return mbar_wait_warp(bar, r.parity, abort_state);
             };
 
-            // score MMAs of tile j out of ring slot `slot` (issued by the elected lane), in two parts so that
-            // the look-ahead for the next tile can run between them
-            auto issue_scores_a = [&](int j, int slot) {
+            // Operand descriptors.  Q and tQ never move: their eight per-k-step descriptors are built once.
+            // Those of a ring slot are built by prepare_*() BEFORE the burst that uses them (while the warp
+            // would be waiting for queue space anyway), so that inside a burst every tcgen05.mma is a single
+            // instruction with its operands ready.
+            uint64_t qd[D / 16], tqd[D / 16];
+#pragma unroll
+            for (int k = 0; k < D / 16; ++k) {
+                const uint32_t koff = ((k / 4) * Plan::kQHalfBytes + (k % 4) * 32) >> 4;
+                qd[k] = make_desc(q_lo + koff);
+                tqd[k] = make_desc(tq_lo + koff);
+            }
+            uint64_t kd[D / 16];            // K-slot descriptors of the score MMAs about to be issued
+            uint64_t vd[kBlockN / 16];      // V-slot descriptors of the value MMAs about to be issued
+            auto prepare_k = [&](int slot) {
                 const uint32_t k_lo = make_desc_lo(smem_ring + slot * Plan::kSlotBytes, 16);
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k)
+                    kd[k] = make_desc(k_lo + (((k / 4) * 2 * Plan::kKvHalfBytes + (k % 4) * 32) >> 4));
+            };
+            auto prepare_v = [&](int slot) {
+                const uint32_t v_lo = make_desc_lo(smem_ring + slot * Plan::kSlotBytes, kVLbo);
+#pragma unroll
+                for (int k = 0; k < kBlockN / 16; ++k) vd[k] = make_desc(v_lo + k * (2048 >> 4));
+            };
+
+            // score MMAs of tile j (issued by the elected lane), in two parts so that the look-ahead for the
+            // next tile can run between them
+            auto issue_scores_a = [&](int j) {
                 const uint32_t tm_s = tmem + kScoreCol0 + (j & 1) * kScoreBufStride;
                 TRACE(21, j);         // MMA: about to issue score MMAs
+                mma_ss<false>(tm_s, qd[0], kd[0], kIdescS1);
 #pragma unroll
-                for (int k = 0; k < D / 16; ++k) {
-                    const uint32_t koff = ((k / 4) * Plan::kQHalfBytes + (k % 4) * 32) >> 4;
-                    const uint32_t boff = ((k / 4) * 2 * Plan::kKvHalfBytes + (k % 4) * 32) >> 4;
-                    mma_ss(tm_s, q_lo + koff, k_lo + boff, kIdescS1, k > 0);
-                }
+                for (int k = 1; k < D / 16; ++k) mma_ss<true>(tm_s, qd[k], kd[k], kIdescS1);
             };
             auto issue_scores_b = [&](int j, int slot) {
-                const uint32_t k_lo = make_desc_lo(smem_ring + slot * Plan::kSlotBytes, 16);
                 const uint32_t tm_ts = tmem + kScoreCol0 + (j & 1) * kScoreBufStride + kBlockN;
                 if (kHasTQ) {
+                    if (kHasTKV) mma_ss<true>(tm_ts, tqd[0], kd[0], kIdescS2);
+                    else mma_ss<false>(tm_ts, tqd[0], kd[0], kIdescS2);
 #pragma unroll
-                    for (int k = 0; k < D / 16; ++k) {
-                        const uint32_t koff = ((k / 4) * Plan::kQHalfBytes + (k % 4) * 32) >> 4;
-                        const uint32_t boff = ((k / 4) * 2 * Plan::kKvHalfBytes + (k % 4) * 32) >> 4;
-                        mma_ss(tm_ts, tq_lo + koff, k_lo + boff, kIdescS2, (kHasTKV || k > 0) ? 1u : 0u);
-                    }
+                    for (int k = 1; k < D / 16; ++k) mma_ss<true>(tm_ts, tqd[k], kd[k], kIdescS2);
                 }
                 tc_commit(smem_u32(&bar_slot_empty[slot]));
                 tc_commit(smem_u32(&bar_s_full[j & 1]));
@@ -521,18 +574,17 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             };
             // value MMAs of tile j out of ring slot `slot`
             auto issue_values = [&](int j, int slot) {
-                const uint32_t v_lo = make_desc_lo(smem_ring + slot * Plan::kSlotBytes, kVLbo);
                 const uint32_t tm_p = tmem + kScoreCol0 + (j & 1) * kScoreBufStride;
                 const uint32_t tm_h = tm_p + kBlockN;
                 TRACE(3, j);          // MMA: about to issue value MMAs
 #pragma unroll
                 for (int k = 0; k < kBlockN / 16; ++k) {
-                    mma_ts(tmem_o, tm_p + k * 8, v_lo + k * (2048 >> 4), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
+                    mma_ts(tmem_o, tm_p + k * 8, vd[k], kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
                 }
                 if (kHasTQ) {
 #pragma unroll
                     for (int k = 0; k < kBlockN / 16; ++k) {
-                        mma_ts(tmem_t, tm_h + k * 8, v_lo + k * (2048 >> 4), kIdescHV, (kHasTKV || j > 0 || k > 0) ? 1u : 0u);
+                        mma_ts(tmem_t, tm_h + k * 8, vd[k], kIdescHV, (kHasTKV || j > 0 || k > 0) ? 1u : 0u);
                     }
                 }
                 tc_commit(smem_u32(&bar_slot_empty[slot]));
@@ -559,14 +611,16 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (ok) ok = wait_full(pos);
             if (ok) {
                 tc_fence_after();
-                if (leader) { issue_scores_a(0, pos.slot); issue_scores_b(0, pos.slot); }
+                prepare_k(pos.slot);
+                if (leader) { issue_scores_a(0); issue_scores_b(0, pos.slot); }
                 __syncwarp();
                 advance(pos);
             }
             if (ok && n_kv > 1) {
                 ok = wait_full(pos);
                 if (ok) {
-                    if (leader) { issue_scores_a(1, pos.slot); issue_scores_b(1, pos.slot); }
+                    prepare_k(pos.slot);
+                    if (leader) { issue_scores_a(1); issue_scores_b(1, pos.slot); }
                     __syncwarp();
                     advance(pos);
                 }
@@ -580,6 +634,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 pos_k = pos;
                 if (has_k) advance(pos);
                 ok = wait_tile(pos_v, pos_k, has_k, 0);
+                prepare_v(pos_v.slot);
+                if (has_k) prepare_k(pos_k.slot);
             }
             for (int j = 0; ok && j < n_kv; ++j) {
                 // ring positions of the next tile
@@ -595,13 +651,18 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 tc_fence_after();
                 if (leader) {
                     issue_values(j, pos_v.slot);
-                    if (has_k) issue_scores_a(j + 2, pos_k.slot);
+                    if (has_k) issue_scores_a(j + 2);
                 }
                 __syncwarp();
                 bool nxt_ready = true;
                 if (nxt_exists) nxt_ready = test_tile(nxt_v, nxt_k, nxt_has_k, j + 1);
                 if (leader && has_k) issue_scores_b(j + 2, pos_k.slot);
                 __syncwarp();
+                // descriptors of the next burst (this warp is held back by the full queue here anyway)
+                if (nxt_exists) {
+                    prepare_v(nxt_v.slot);
+                    if (nxt_has_k) prepare_k(nxt_k.slot);
+                }
                 if (nxt_exists && !nxt_ready) ok = wait_tile(nxt_v, nxt_k, nxt_has_k, j + 1);
                 pos_v = nxt_v;
                 pos_k = nxt_k;
@@ -621,7 +682,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         // lane) and columns [32*half, 32*half + 32) of every score tile, half = (w - 2) / 4.
         // =====================================================================================
         const int half = (warp - kFirstSoftmaxWarp) >> 2;
-        const int row = (warp & 3) * 32 + lane;                       // 0..127: a warp may only touch lanes 32*(warp%4)..+31
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;                          // 0..127: a warp may only touch lanes 32*(warp%4)..+31
         const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
         const float c1 = args.scale_log2;
         const float sc = args.scale;
@@ -673,8 +735,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             mx *= c1;    // -inf when the whole half is masked (c1 == 0 gives NaN, which fmaxf below drops)
             // exchange with the thread that owns the other half of this row
             xchg_max[bsel][half][row] = mx;
-            mbar_arrive(smem_u32(&bar_xchg[bsel]));
-            if (!mbar_wait_warp(smem_u32(&bar_xchg[bsel]), (j >> 1) & 1, abort_state)) { ok = false; break; }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_xchg[bsel][quarter]));
+            if (!mbar_wait_warp(smem_u32(&bar_xchg[bsel][quarter]), (j >> 1) & 1, abort_state)) { ok = false; break; }
             mx = fmaxf(mx, xchg_max[bsel][half ^ 1][row]);
 
             // m_new = max(m, rowmax), applied lazily: the result does not depend on which
@@ -704,14 +767,22 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             l_run *= alpha;
             r_run *= alpha;
 
-            // P~ = exp(S - m_new), l += rowsum(P~)
-            float ls4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+            // P~ = exp(S - m_new), l += rowsum(P~)   (two columns per FMA-pipe instruction)
+            const uint64_t c1c1 = pack_f32x2(c1, c1);
+            const uint64_t negm = pack_f32x2(-m_ref, -m_ref);
+            uint64_t ls2[2] = {0ull, 0ull};     // (+0.0f, +0.0f)
 #pragma unroll
-            for (int c = 0; c < kHalfN; ++c) {
-                const float p = ex2f(fmaf(__uint_as_float(sv[c]), c1, -m_ref));
-                sv[c] = __float_as_uint(p);
-                ls4[c & 3] += p;
+            for (int c = 0; c < kHalfN; c += 2) {
+                float x0, x1;
+                unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), c1c1, negm), x0, x1);
+                const float p0 = ex2f(x0), p1 = ex2f(x1);
+                sv[c] = __float_as_uint(p0);
+                sv[c + 1] = __float_as_uint(p1);
+                ls2[(c >> 1) & 1] = add_f32x2(ls2[(c >> 1) & 1], pack_f32x2(p0, p1));
             }
+            float ls4[4];
+            unpack_f32x2(ls2[0], ls4[0], ls4[1]);
+            unpack_f32x2(ls2[1], ls4[2], ls4[3]);
             if (valid < kHalfN) {
                 // exact zeros for masked keys whatever the scale (0 * inf above would give NaN)
                 ls4[0] = ls4[1] = ls4[2] = ls4[3] = 0.0f;
@@ -747,8 +818,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     tmem_st2(tm_s + kHalfN + 2 * half, num_h, lsum);
                     tc_wait_st();
                     tc_fence_before();
-                    mbar_arrive(smem_u32(&bar_xchg[2]));
-                    if (!mbar_wait_warp(smem_u32(&bar_xchg[2]), 0, abort_state)) { ok = false; break; }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bar_xchg[2][quarter]));
+                    if (!mbar_wait_warp(smem_u32(&bar_xchg[2][quarter]), 0, abort_state)) { ok = false; break; }
                     tc_fence_after();
                     tmem_ld2(tm_s + kHalfN + 2 * (half ^ 1), num_o, lsum_o);
                     tc_wait_ld();
@@ -756,14 +828,25 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     ts_shift = half == 0 ? (num_h + num_o) / (lsum + lsum_o) : (num_o + num_h) / (lsum_o + lsum);
                 }
                 // H~ = P~ . tS, r += rowsum(H~)
-                float rs4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                const uint64_t scsc = pack_f32x2(sc, sc);
+                const uint64_t negshift = pack_f32x2(-ts_shift, -ts_shift);
+                uint64_t rs2[2] = {0ull, 0ull};
 #pragma unroll
-                for (int c = 0; c < kHalfN; ++c) {
-                    const float hv = __uint_as_float(sv[c]) * fmaf(__uint_as_float(tv[c]), sc, -ts_shift);
-                    tv[c] = __float_as_uint(hv);
-                    rs4[c & 3] += hv;
+                for (int c = 0; c < kHalfN; c += 2) {
+                    const uint64_t ts2 = fma_f32x2(pack_f32x2(__uint_as_float(tv[c]), __uint_as_float(tv[c + 1])), scsc, negshift);
+                    const uint64_t h2 = mul_f32x2(pack_f32x2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), ts2);
+                    float h0, h1;
+                    unpack_f32x2(h2, h0, h1);
+                    tv[c] = __float_as_uint(h0);
+                    tv[c + 1] = __float_as_uint(h1);
+                    rs2[(c >> 1) & 1] = add_f32x2(rs2[(c >> 1) & 1], h2);
                 }
-                r_run += (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
+                {
+                    float a0, a1, a2, a3;
+                    unpack_f32x2(rs2[0], a0, a1);
+                    unpack_f32x2(rs2[1], a2, a3);
+                    r_run += (a0 + a1) + (a2 + a3);
+                }
                 uint32_t pk[kHalfN / 2];
 #pragma unroll
                 for (int c = 0; c < kHalfN / 2; ++c) pk[c] = pack_bf16(__uint_as_float(tv[2 * c]), __uint_as_float(tv[2 * c + 1]));
@@ -771,7 +854,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             }
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(smem_u32(&bar_p_full[bsel]));
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_p_full[bsel]));
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
             if (trace_me && j < kTraceSteps) g_trace[13 + (warp - kFirstSoftmaxWarp)][j] = clock64();    // softmax warp: arrived
 #endif
@@ -790,8 +874,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             tmem_st2(tm_x + 2 * half, l_run, r_run);
             tc_wait_st();
             tc_fence_before();
-            mbar_arrive(smem_u32(&bar_xchg[2]));
-            ok = mbar_wait_warp(smem_u32(&bar_xchg[2]), kHasTQ ? 1 : 0, abort_state);   // phase 0 was the first-tile exchange
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_xchg[2][quarter]));
+            ok = mbar_wait_warp(smem_u32(&bar_xchg[2][quarter]), kHasTQ ? 1 : 0, abort_state);   // phase 0 was the first-tile exchange
         }
         if (ok) {
             tc_fence_after();
