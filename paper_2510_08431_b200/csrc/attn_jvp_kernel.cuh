@@ -1,16 +1,17 @@
 // Attention-JVP forward kernel for sm_100a (Algorithm 2: FlashAttention-2 forward with JVP).
 //
 // One CTA owns a 128-row query tile of one (batch, head) and streams the keys in
-// tiles of 64.  Roles (warp-specialised, 320 threads):
-//   warp 0     MMA issuer (one thread): tcgen05.mma with accumulators in tensor memory.
+// tiles of 64.  Roles (warp-specialised, 64 + 128*kGroups threads):
+//   warp 0     MMA issuer: the whole warp runs the loop in lock step, one elected lane issues
+//              tcgen05.mma with accumulators in tensor memory.
 //   warp 1     TMA producer: Q,tQ once, then K|tK and V|tV tiles into a shared-memory ring.
-//   warps 2-9  softmax: two groups of four warps; thread (w, lane) owns query row 32*(w%4) + lane
-//              and the 32-column half (w-2)/4 of every score tile.  Reads S and tS from tensor memory,
-//              keeps m, l, r (Algorithm 2 lines 10-12, 16) in registers (l, r as per-half
-//              partial sums; the row max is exchanged through shared memory), writes
-//              P~ and H~ = P~ . tS back to tensor memory as bf16 MMA operands,
-//              rescales the accumulators when the running max moves, and runs
-//              the epilogue (lines 19-23).
+//   warps 2..  softmax: kGroups groups of four warps; thread (w, lane) owns query row
+//              32*(w%4) + lane (its tensor-memory lane) and 64/kGroups columns of every score tile.
+//              Reads S and tS from tensor memory, keeps m, l, r (Algorithm 2 lines 10-12, 16) in
+//              registers, writes P~ and H~ = P~ . tS back to tensor memory as bf16 MMA operands,
+//              rescales the accumulators when the running max moves, and runs the epilogue
+//              (lines 19-23).  With kGroups = 2 the two owners of a row exchange the row max through
+//              shared memory and their partial sums through dead tensor-memory columns.
 //
 // Tensor-memory map (512 columns x 128 lanes, fp32):
 //   [0, D)        O  accumulator (line 13)
@@ -35,12 +36,16 @@ namespace attn_jvp {
 
 constexpr int kBlockM = 128;        // query rows per CTA (B_r)
 constexpr int kBlockN = 64;         // keys per tile (B_c)
-constexpr int kSoftmaxThreads = 256;   // two warpgroups, each owning 32 of the 64 columns of a score tile
+#ifndef ATTN_JVP_SOFTMAX_GROUPS
+#define ATTN_JVP_SOFTMAX_GROUPS 1     // measured: one group of four warps is as fast as two and needs no exchange
+#endif
+constexpr int kGroups = ATTN_JVP_SOFTMAX_GROUPS;   // groups of four softmax warps; each owns 64/kGroups columns of a score tile
+constexpr int kSoftmaxThreads = 128 * kGroups;
 constexpr int kMmaWarp = 0;            // the two single-thread roles come first (oldest warps of the CTA)
 constexpr int kProducerWarp = 1;
 constexpr int kFirstSoftmaxWarp = 2;
 constexpr int kThreads = kSoftmaxThreads + 64;
-constexpr int kHalfN = kBlockN / 2;
+constexpr int kHalfN = kBlockN / kGroups;      // score columns per softmax thread
 constexpr int kTmemCols = 512;
 constexpr int kScoreCol0 = 256;     // first column of score buffer 0
 constexpr int kScoreBufStride = 128;
@@ -707,8 +712,11 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
             uint32_t sv[kHalfN];
             uint32_t tv[kHalfN];
-            TMEM_LD32(tm_s + half * kHalfN, sv, 0);
-            if (kHasTQ) TMEM_LD32(tm_ts + half * kHalfN, tv, 0);
+#pragma unroll
+            for (int c0 = 0; c0 < kHalfN; c0 += 32) {
+                TMEM_LD32(tm_s + half * kHalfN + c0, sv, c0);
+                if (kHasTQ) TMEM_LD32(tm_ts + half * kHalfN + c0, tv, c0);
+            }
             tc_wait_ld();
 
             // keys past Lk (zero-filled by TMA) must not enter the softmax
@@ -733,12 +741,14 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             float mx = neg_scale ? fminf(fminf(mx4[0], mx4[1]), fminf(mx4[2], mx4[3]))
                                  : fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
             mx *= c1;    // -inf when the whole half is masked (c1 == 0 gives NaN, which fmaxf below drops)
-            // exchange with the thread that owns the other half of this row
-            xchg_max[bsel][half][row] = mx;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bar_xchg[bsel][quarter]));
-            if (!mbar_wait_warp(smem_u32(&bar_xchg[bsel][quarter]), (j >> 1) & 1, abort_state)) { ok = false; break; }
-            mx = fmaxf(mx, xchg_max[bsel][half ^ 1][row]);
+            if (kGroups == 2) {
+                // exchange with the thread that owns the other half of this row
+                xchg_max[bsel][half][row] = mx;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bar_xchg[bsel][quarter]));
+                if (!mbar_wait_warp(smem_u32(&bar_xchg[bsel][quarter]), (j >> 1) & 1, abort_state)) { ok = false; break; }
+                mx = fmaxf(mx, xchg_max[bsel][half ^ 1][row]);
+            }
 
             // m_new = max(m, rowmax), applied lazily: the result does not depend on which
             // reference is used as long as exp() stays in range.  Both owners of a row take
@@ -755,7 +765,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 tc_fence_after();
                 constexpr int kAccCols = kHasTQ ? 2 * D : D;     // each half rescales its share of the columns
 #pragma unroll 1
-                for (int c0 = half * (kAccCols / 2); c0 < (half + 1) * (kAccCols / 2); c0 += 32) {
+                for (int c0 = half * (kAccCols / kGroups); c0 < (half + 1) * (kAccCols / kGroups); c0 += 32) {
                     uint32_t acc[32];
                     TMEM_LD32(tmem_o + lane_base + c0, acc, 0);
                     tc_wait_ld();
@@ -798,7 +808,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 uint32_t pk[kHalfN / 2];
 #pragma unroll
                 for (int c = 0; c < kHalfN / 2; ++c) pk[c] = pack_bf16(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1]));
-                TMEM_ST16(tm_s + half * (kHalfN / 2), pk, 0);
+#pragma unroll
+                for (int c0 = 0; c0 < kHalfN / 2; c0 += 16) TMEM_ST16(tm_s + half * (kHalfN / 2) + c0, pk, c0);
             }
             if (kHasTQ) {
                 // tO does not change when a per-row constant is subtracted from tS (softmax is shift
@@ -814,18 +825,22 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     // 32.. of the S buffer are dead once both have loaded their scores (the exchange of
                     // the maxima above guarantees that) and both threads address the same lane.
                     const float num_h = (nm4[0] + nm4[1]) + (nm4[2] + nm4[3]);
-                    float num_o, lsum_o;
-                    tmem_st2(tm_s + kHalfN + 2 * half, num_h, lsum);
-                    tc_wait_st();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&bar_xchg[2][quarter]));
-                    if (!mbar_wait_warp(smem_u32(&bar_xchg[2][quarter]), 0, abort_state)) { ok = false; break; }
-                    tc_fence_after();
-                    tmem_ld2(tm_s + kHalfN + 2 * (half ^ 1), num_o, lsum_o);
-                    tc_wait_ld();
-                    // same operand order in both threads, so that both get the same bits
-                    ts_shift = half == 0 ? (num_h + num_o) / (lsum + lsum_o) : (num_o + num_h) / (lsum_o + lsum);
+                    if (kGroups == 2) {
+                        float num_o, lsum_o;
+                        tmem_st2(tm_s + kBlockN / 2 + 2 * half, num_h, lsum);
+                        tc_wait_st();
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&bar_xchg[2][quarter]));
+                        if (!mbar_wait_warp(smem_u32(&bar_xchg[2][quarter]), 0, abort_state)) { ok = false; break; }
+                        tc_fence_after();
+                        tmem_ld2(tm_s + kBlockN / 2 + 2 * (half ^ 1), num_o, lsum_o);
+                        tc_wait_ld();
+                        // same operand order in both threads, so that both get the same bits
+                        ts_shift = half == 0 ? (num_h + num_o) / (lsum + lsum_o) : (num_o + num_h) / (lsum_o + lsum);
+                    } else {
+                        ts_shift = num_h / lsum;
+                    }
                 }
                 // H~ = P~ . tS, r += rowsum(H~)
                 const uint64_t scsc = pack_f32x2(sc, sc);
@@ -850,7 +865,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 uint32_t pk[kHalfN / 2];
 #pragma unroll
                 for (int c = 0; c < kHalfN / 2; ++c) pk[c] = pack_bf16(__uint_as_float(tv[2 * c]), __uint_as_float(tv[2 * c + 1]));
-                TMEM_ST16(tm_ts + half * (kHalfN / 2), pk, 0);
+#pragma unroll
+                for (int c0 = 0; c0 < kHalfN / 2; c0 += 16) TMEM_ST16(tm_ts + half * (kHalfN / 2) + c0, pk, c0);
             }
             tc_wait_st();
             tc_fence_before();
@@ -866,11 +882,11 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         // tile n-2 may still be running here: wait for them first, then for those of tile n-1.
         if (ok && n_kv >= 2) ok = mbar_wait_warp(smem_u32(&bar_pv_done), (n_kv - 2) & 1, abort_state);
         if (ok) ok = mbar_wait_warp(smem_u32(&bar_pv_done), (n_kv - 1) & 1, abort_state);
-        if (ok) {
+        if (ok && kGroups == 2) {
             // total l and r of the row = sum of the two halves' shares, swapped through the (now dead)
             // score columns of tensor memory.
             tc_fence_after();
-            const uint32_t tm_x = tmem + lane_base + kScoreCol0 + kHalfN;
+            const uint32_t tm_x = tmem + lane_base + kScoreCol0 + kBlockN / 2;
             tmem_st2(tm_x + 2 * half, l_run, r_run);
             tc_wait_st();
             tc_fence_before();
@@ -880,11 +896,14 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         if (ok) {
             tc_fence_after();
-            float l_o, r_o;
-            tmem_ld2(tmem + lane_base + kScoreCol0 + kHalfN + 2 * (half ^ 1), l_o, r_o);
-            tc_wait_ld();
-            const float l_tot = half == 0 ? l_run + l_o : l_o + l_run;
-            const float r_tot = half == 0 ? r_run + r_o : r_o + r_run;
+            float l_tot = l_run, r_tot = r_run;
+            if (kGroups == 2) {
+                float l_o, r_o;
+                tmem_ld2(tmem + lane_base + kScoreCol0 + kBlockN / 2 + 2 * (half ^ 1), l_o, r_o);
+                tc_wait_ld();
+                l_tot = half == 0 ? l_run + l_o : l_o + l_run;
+                r_tot = half == 0 ? r_run + r_o : r_o + r_run;
+            }
             const int qi = q0 + row;
             const bool in_range = qi < args.Lq;
             const float inv_l = 1.0f / l_tot;
@@ -893,7 +912,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             __nv_bfloat16* o_row = args.o + row_off;
             __nv_bfloat16* to_row = kHasTQ ? args.to + row_off : nullptr;
 #pragma unroll 1
-            for (int c0 = half * (D / 2); c0 < (half + 1) * (D / 2); c0 += 32) {
+            for (int c0 = half * (D / kGroups); c0 < (half + 1) * (D / kGroups); c0 += 32) {
                 uint32_t ov[32];
                 uint32_t tvv[32];
                 TMEM_LD32(tmem_o + lane_base + c0, ov, 0);
