@@ -16,8 +16,8 @@
  *
  * Conventions common to every entry point
  *   - All tensor pointers are DEVICE pointers owned by the caller.  The
- *     library neither frees nor retains them, allocates no device memory and
- *     needs no workspace.
+ *     library neither frees nor retains them and allocates no device memory;
+ *     only the split-KV entry point needs a (caller-provided) workspace.
  *   - q, tq, o, to : bf16, layout [B][Lq][H][D] contiguous ("BLHD").
  *     k, v, tk, tv : bf16, layout [B][Lk][H][D] contiguous.
  *     lse          : fp32, layout [B][H][Lq], natural log of the scaled scores.
@@ -60,6 +60,7 @@ extern "C" {
 #define ATTN_JVP_ERR_CUDA            9  /* a CUDA runtime / driver call failed (see strerror) */
 #define ATTN_JVP_ERR_DEVICE_TIMEOUT 10  /* a bounded device-side wait expired */
 #define ATTN_JVP_ERR_DEVICE_LAYOUT  11  /* the kernel's shared-memory layout did not fit (reported like a timeout) */
+#define ATTN_JVP_ERR_WORKSPACE      12  /* split-KV workspace too small */
 
 /*
  * attn_jvp_fwd -- O, tO and LSE of Algorithm 2 in one pass, on the stream set
@@ -84,6 +85,40 @@ int attn_jvp_fwd_stream(const void* q, const void* k, const void* v,
                         void* o, void* to, float* lse,
                         int B, int H, int Lq, int Lk, int D,
                         float scale, unsigned flags, void* cuda_stream);
+
+/*
+ * attn_jvp_fwd_mu -- Algorithm 2 plus one more per-row side output, mu = rowsum(P . tS) (the r / l of
+ * Algorithm 2 lines 16 and 21, i.e. the tangent of L = LSE).  mu: device, fp32 [B][H][Lq], required.
+ * Everything else as attn_jvp_fwd_stream.  With ATTN_JVP_FWD_ONLY mu is written as 0.
+ */
+int attn_jvp_fwd_mu(const void* q, const void* k, const void* v,
+                    const void* tq, const void* tk, const void* tv,
+                    void* o, void* to, float* lse, float* mu,
+                    int B, int H, int Lq, int Lk, int D,
+                    float scale, unsigned flags, void* cuda_stream);
+
+/*
+ * Split-KV variant for few queries and many keys: the keys are cut into chunks of whole 64-key tiles,
+ * each (query tile, head, chunk) runs Algorithm 2 on its chunk, and a second kernel merges the chunks.
+ * With per-chunk results (O_c, tO_c, LSE_c, mu_c) and w_c = exp(LSE_c - LSE), LSE = log sum_c exp(LSE_c):
+ *     O = sum_c w_c O_c,  mu = sum_c w_c mu_c,  tO = sum_c w_c (tO_c + mu_c O_c) - mu O,
+ * which is the aggregated form of Appendix C.1 regrouped by chunk (exact in real arithmetic).
+ *
+ *   splits           requested number of chunks (>= 1); the library uses ceil(tiles / ceil(tiles / splits))
+ *                    chunks so that none is empty; 1 chunk = the plain kernel, no workspace needed.
+ *   workspace        device scratch owned by the caller, 16-byte aligned, at least
+ *                    attn_jvp_splitkv_workspace_bytes(...) bytes; contents undefined afterwards.  Calls
+ *                    that share a workspace must not overlap on the GPU.
+ *   mu               optional (may be NULL).  Other arguments as attn_jvp_fwd_stream.
+ * Returns ATTN_JVP_ERR_WORKSPACE if workspace_bytes is too small.
+ */
+size_t attn_jvp_splitkv_workspace_bytes(int B, int H, int Lq, int Lk, int D, int splits);
+int attn_jvp_fwd_splitkv(const void* q, const void* k, const void* v,
+                         const void* tq, const void* tk, const void* tv,
+                         void* o, void* to, float* lse, float* mu,
+                         int B, int H, int Lq, int Lk, int D,
+                         float scale, unsigned flags, int splits,
+                         void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* Sets the stream attn_jvp_fwd launches on for the calling host thread
  * (thread-local; NULL = legacy default stream).  Always returns 0. */

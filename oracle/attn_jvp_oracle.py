@@ -153,3 +153,22 @@ def attn_jvp_def_bf16_rows(q, k, v, tq, tk, tv, B, H, Lq, Lk, D, scale, rows):
     inv = np.empty_like(order)
     inv[order] = np.arange(n)
     return O[inv], tO[inv], LSE[inv], MU[inv]
+
+
+def splitkv_merge(O_c, tO_c, LSE_c, MU_c):
+    """Merges per-chunk results of a split over the keys (fp64 numpy; test infrastructure).
+
+    Chunk c gave (O_c, tO_c, LSE_c, mu_c), each normalised within the chunk.  The full softmax weights are
+    P_j = w_c P^c_j with w_c = exp(LSE_c - LSE), LSE = log sum_c exp(LSE_c), so from the aggregated form of
+    Appendix C.1 (tO = (P.tS) V + P tV - diag(mu) O):
+        O = sum_c w_c O_c,  mu = sum_c w_c mu_c,  tO = sum_c w_c (tO_c + mu_c O_c) - mu O.
+    Inputs are lists over chunks of arrays [n][D], [n][D], [n], [n].  Returns (O, tO, LSE, mu).
+    """
+    L = np.stack(LSE_c)                      # [C][n]
+    m = L.max(axis=0)
+    LSE = m + np.log(np.exp(L - m).sum(axis=0))
+    w = np.exp(L - LSE)                      # [C][n]
+    O = sum(w[c][:, None] * O_c[c] for c in range(len(O_c)))
+    mu = sum(w[c] * MU_c[c] for c in range(len(O_c)))
+    tO = sum(w[c][:, None] * (tO_c[c] + MU_c[c][:, None] * O_c[c]) for c in range(len(O_c))) - mu[:, None] * O
+    return O, tO, LSE, mu

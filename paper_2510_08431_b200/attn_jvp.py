@@ -17,10 +17,11 @@ KV_TANGENT_FREE = 0x1
 FWD_ONLY = 0x2
 
 ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED_D, ERR_ALIGN, ERR_FLAGS = 1, 2, 3, 4, 5
-ERR_SCALE, ERR_ALIAS, ERR_ARCH, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_DEVICE_LAYOUT = 6, 7, 8, 9, 10, 11
+ERR_SCALE, ERR_ALIAS, ERR_ARCH, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_DEVICE_LAYOUT, ERR_WORKSPACE = 6, 7, 8, 9, 10, 11, 12
 
-EXPORTS = ("attn_jvp_fwd", "attn_jvp_fwd_stream", "attn_jvp_set_stream", "attn_jvp_device_status",
-           "attn_jvp_strerror", "attn_jvp_version")
+EXPORTS = ("attn_jvp_fwd", "attn_jvp_fwd_stream", "attn_jvp_fwd_mu", "attn_jvp_splitkv_workspace_bytes",
+           "attn_jvp_fwd_splitkv", "attn_jvp_set_stream", "attn_jvp_device_status", "attn_jvp_strerror",
+           "attn_jvp_version")
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libattn_jvp.so")
 _lock = threading.Lock()
@@ -53,6 +54,12 @@ def load():
             lib.attn_jvp_fwd.restype = ci
             lib.attn_jvp_fwd_stream.argtypes = common + [vp]
             lib.attn_jvp_fwd_stream.restype = ci
+            lib.attn_jvp_fwd_mu.argtypes = [vp] * 10 + [ci] * 5 + [cf, cu, vp]
+            lib.attn_jvp_fwd_mu.restype = ci
+            lib.attn_jvp_splitkv_workspace_bytes.argtypes = [ci] * 6
+            lib.attn_jvp_splitkv_workspace_bytes.restype = ctypes.c_size_t
+            lib.attn_jvp_fwd_splitkv.argtypes = [vp] * 10 + [ci] * 5 + [cf, cu, ci, vp, ctypes.c_size_t, vp]
+            lib.attn_jvp_fwd_splitkv.restype = ci
             lib.attn_jvp_set_stream.argtypes = [vp]
             lib.attn_jvp_set_stream.restype = ci
             lib.attn_jvp_device_status.argtypes = []
@@ -101,17 +108,39 @@ def attn_jvp_fwd_stream(q, k, v, tq, tk, tv, o, to, lse, B, H, Lq, Lk, D, scale,
                                           _ptr(cuda_stream)))
 
 
+def attn_jvp_fwd_mu(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, Lk, D, scale, flags, cuda_stream) -> int:
+    return int(load().attn_jvp_fwd_mu(_ptr(q), _ptr(k), _ptr(v), _ptr(tq), _ptr(tk), _ptr(tv), _ptr(o), _ptr(to),
+                                      _ptr(lse), _ptr(mu), B, H, Lq, Lk, D, float(scale), int(flags),
+                                      _ptr(cuda_stream)))
+
+
+def attn_jvp_splitkv_workspace_bytes(B, H, Lq, Lk, D, splits) -> int:
+    return int(load().attn_jvp_splitkv_workspace_bytes(B, H, Lq, Lk, D, splits))
+
+
+def attn_jvp_fwd_splitkv(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, Lk, D, scale, flags, splits, workspace,
+                         workspace_bytes, cuda_stream) -> int:
+    return int(load().attn_jvp_fwd_splitkv(_ptr(q), _ptr(k), _ptr(v), _ptr(tq), _ptr(tk), _ptr(tv), _ptr(o),
+                                           _ptr(to), _ptr(lse), _ptr(mu), B, H, Lq, Lk, D, float(scale), int(flags),
+                                           int(splits), _ptr(workspace), int(workspace_bytes), _ptr(cuda_stream)))
+
+
 def _check(t, name, shape):
     if not t.is_cuda or t.dtype != torch.bfloat16 or tuple(t.shape) != shape or not t.is_contiguous():
         raise ValueError(f"{name} must be a contiguous CUDA bf16 tensor of shape {shape}")
 
 
-def attention_jvp(q, k, v, tq=None, tk=None, tv=None, scale=None, fwd_only=False, out=None):
+def attention_jvp(q, k, v, tq=None, tk=None, tv=None, scale=None, fwd_only=False, out=None,
+                  return_mu=False, splits=1, workspace=None):
     """O, tO, LSE of Algorithm 2 for [B][L][H][D] bf16 CUDA tensors, on torch's current stream.
 
     ``tk is None and tv is None`` selects the tangent-free K/V path (cross-attention on a constant
     context); ``fwd_only`` runs the plain forward (returns tO = None).  ``out`` may supply
-    preallocated (o, to, lse).  Returns (o, to, lse).
+    preallocated (o, to, lse).  ``return_mu`` adds mu = rowsum(P . tS) (the tangent of LSE) as a fourth
+    result.  ``splits`` > 1 cuts the keys into chunks processed by independent CTAs and merged by a
+    second kernel (for few queries and many keys); ``workspace`` may supply its scratch (a CUDA uint8
+    tensor of at least attn_jvp_splitkv_workspace_bytes), else it is allocated here with torch.
+    Returns (o, to, lse) or (o, to, lse, mu).
     """
     B, Lq, H, D = q.shape
     Lk = k.shape[1]
@@ -134,12 +163,23 @@ def attention_jvp(q, k, v, tq=None, tk=None, tv=None, scale=None, fwd_only=False
         lse = torch.empty((B, H, Lq), dtype=torch.float32, device=q.device)
     else:
         o, to, lse = out
+    mu = torch.empty((B, H, Lq), dtype=torch.float32, device=q.device) if return_mu else None
     with torch.cuda.device(q.device):
         stream = torch.cuda.current_stream().cuda_stream
-        rc = attn_jvp_fwd_stream(q, k, v, tq, tk, tv, o, to, lse, B, H, Lq, Lk, D, scale, flags, stream)
+        if splits > 1:
+            need = attn_jvp_splitkv_workspace_bytes(B, H, Lq, Lk, D, splits)
+            if workspace is None and need > 0:
+                workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+            nbytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+            rc = attn_jvp_fwd_splitkv(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, Lk, D, scale, flags, splits,
+                                      workspace, nbytes, stream)
+        elif return_mu:
+            rc = attn_jvp_fwd_mu(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, Lk, D, scale, flags, stream)
+        else:
+            rc = attn_jvp_fwd_stream(q, k, v, tq, tk, tv, o, to, lse, B, H, Lq, Lk, D, scale, flags, stream)
     if rc != 0:
         raise AttnJvpError(rc, attn_jvp_strerror(rc))
-    return o, to, lse
+    return (o, to, lse, mu) if return_mu else (o, to, lse)
 
 
 def attention_jvp_host(q, k, v, tq=None, tk=None, tv=None, scale=None, fwd_only=False, device="cuda:0"):

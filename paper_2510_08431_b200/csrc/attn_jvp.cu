@@ -22,7 +22,7 @@ thread_local char tl_strerror_buf[384];
 
 int* g_host_status[kMaxDevices] = {};       // mapped pinned host words, one per device
 int* g_host_status_dev[kMaxDevices] = {};   // their device-side addresses
-int g_dyn_smem[kMaxDevices][2][3] = {};     // dynamic shared memory per kernel instantiation, 0 = not set up
+int g_dyn_smem[kMaxDevices][2][3][2] = {};  // dynamic shared memory per kernel instantiation, 0 = not set up
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -71,10 +71,10 @@ bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
     return a0 < b0 + nb && b0 < a0 + na;
 }
 
-template <int D, int MODE>
+template <int D, int MODE, bool SPLIT>
 int launch(const CUtensorMap* maps, const KernelArgs& ka, dim3 grid, cudaStream_t stream, int dev) {
-    auto kern = attn_jvp::attn_jvp_fwd_kernel<D, MODE>;
-    int& smem = g_dyn_smem[dev][D == 128][MODE];
+    auto kern = attn_jvp::attn_jvp_fwd_kernel<D, MODE, SPLIT>;
+    int& smem = g_dyn_smem[dev][D == 128][MODE][SPLIT];
     if (smem == 0) {
         // dynamic shared memory = the operand layout plus slack for its 1024-byte alignment, capped by
         // what the device leaves after the kernel's static shared memory
@@ -102,9 +102,32 @@ int launch(const CUtensorMap* maps, const KernelArgs& ka, dim3 grid, cudaStream_
     return 0;
 }
 
+// Bytes of scratch the split-KV path needs: per chunk fp32 O and tO partials ([B][Lq][H][D]) and fp32 LSE and mu
+// partials ([B][H][Lq], each padded to a multiple of 16 bytes).
+struct SplitLayout {
+    size_t vec_bytes;    // one chunk set of O (or tO) partials, all chunks
+    size_t stat_bytes;   // one chunk set of LSE (or mu) partials, all chunks, padded
+    size_t total;
+};
+SplitLayout split_layout(int B, int H, int Lq, int D, int splits) {
+    SplitLayout L;
+    L.vec_bytes = (size_t)splits * B * Lq * H * D * sizeof(float);
+    L.stat_bytes = (((size_t)splits * B * H * Lq * sizeof(float)) + 15) & ~(size_t)15;
+    L.total = 2 * L.vec_bytes + 2 * L.stat_bytes;
+    return L;
+}
+// Chunks actually used for `splits` requested chunks: whole 64-key tiles per chunk, no empty chunk.
+void split_plan(int Lk, int splits, int* tiles_per_split, int* eff_splits) {
+    const int n_tiles = (Lk + attn_jvp::kBlockN - 1) / attn_jvp::kBlockN;
+    if (splits > n_tiles) splits = n_tiles;
+    const int tps = (n_tiles + splits - 1) / splits;
+    *tiles_per_split = tps;
+    *eff_splits = (n_tiles + tps - 1) / tps;
+}
+
 int run(const void* q, const void* k, const void* v, const void* tq, const void* tk, const void* tv,
-        void* o, void* to, float* lse, int B, int H, int Lq, int Lk, int D, float scale, unsigned flags,
-        cudaStream_t stream) {
+        void* o, void* to, float* lse, float* mu, int B, int H, int Lq, int Lk, int D, float scale, unsigned flags,
+        int splits, void* workspace, size_t workspace_bytes, cudaStream_t stream) {
     // ---- validation: nothing is enqueued unless everything checks out ----
     if (flags & ~(ATTN_JVP_KV_TANGENT_FREE | ATTN_JVP_FWD_ONLY)) return ATTN_JVP_ERR_FLAGS;
     const bool fwd_only = (flags & ATTN_JVP_FWD_ONLY) != 0;
@@ -119,19 +142,30 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     if (!fwd_only && (!tq || !to)) return ATTN_JVP_ERR_NULL;
     if (mode == attn_jvp::kModeJvp && (!tk || !tv)) return ATTN_JVP_ERR_NULL;
     if (!std::isfinite(scale)) return ATTN_JVP_ERR_SCALE;
+    if (splits < 1 || splits > 1024) return ATTN_JVP_ERR_SHAPE;
+    int tiles_per_split = 0, eff_splits = 1;
+    split_plan(Lk, splits, &tiles_per_split, &eff_splits);
+    const bool split = eff_splits > 1;
+    SplitLayout lay = split_layout(B, H, Lq, D, eff_splits);
+    if (split) {
+        if (!workspace) return ATTN_JVP_ERR_NULL;
+        if ((uintptr_t)workspace & 15u) return ATTN_JVP_ERR_ALIGN;
+        if (workspace_bytes < lay.total) return ATTN_JVP_ERR_WORKSPACE;
+        if ((long long)B * eff_splits > 65535) return ATTN_JVP_ERR_SHAPE;
+    }
     const void* used_in[6] = {q, k, v, fwd_only ? nullptr : tq, mode == attn_jvp::kModeJvp ? tk : nullptr,
                               mode == attn_jvp::kModeJvp ? tv : nullptr};
-    void* used_out[3] = {o, fwd_only ? nullptr : to, lse};
+    void* used_out[5] = {o, fwd_only ? nullptr : to, lse, mu, split ? workspace : nullptr};
     for (const void* p : used_in) if (p && ((uintptr_t)p & 15u)) return ATTN_JVP_ERR_ALIGN;
     for (const void* p : used_out) if (p && ((uintptr_t)p & 15u)) return ATTN_JVP_ERR_ALIGN;
     const size_t q_bytes = (size_t)B * Lq * H * D * 2, k_bytes = (size_t)B * Lk * H * D * 2;
     const size_t lse_bytes = (size_t)B * H * Lq * 4;
     const size_t in_bytes[6] = {q_bytes, k_bytes, k_bytes, q_bytes, k_bytes, k_bytes};
-    const size_t out_bytes[3] = {q_bytes, q_bytes, lse_bytes};
-    for (int a = 0; a < 3; ++a) {
+    const size_t out_bytes[5] = {q_bytes, q_bytes, lse_bytes, lse_bytes, lay.total};
+    for (int a = 0; a < 5; ++a) {
         for (int i = 0; i < 6; ++i)
             if (overlaps(used_out[a], out_bytes[a], used_in[i], in_bytes[i])) return ATTN_JVP_ERR_ALIAS;
-        for (int c = a + 1; c < 3; ++c)
+        for (int c = a + 1; c < 5; ++c)
             if (overlaps(used_out[a], out_bytes[a], used_out[c], out_bytes[c])) return ATTN_JVP_ERR_ALIAS;
     }
 
@@ -177,20 +211,48 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     ka.n_kv_tiles = (Lk + attn_jvp::kBlockN - 1) / attn_jvp::kBlockN;
     ka.scale = scale;
     ka.scale_log2 = scale * 1.4426950408889634f;
+    ka.mu = mu;
+    ka.B = B;
+    ka.splits = eff_splits;
+    ka.tiles_per_split = tiles_per_split;
+    ka.part_o = ka.part_to = ka.part_lse = ka.part_mu = nullptr;
+    if (split) {
+        char* w = static_cast<char*>(workspace);
+        ka.part_o = reinterpret_cast<float*>(w);
+        ka.part_to = reinterpret_cast<float*>(w + lay.vec_bytes);
+        ka.part_lse = reinterpret_cast<float*>(w + 2 * lay.vec_bytes);
+        ka.part_mu = reinterpret_cast<float*>(w + 2 * lay.vec_bytes + lay.stat_bytes);
+    }
 
-    const dim3 grid((Lq + attn_jvp::kBlockM - 1) / attn_jvp::kBlockM, H, B);
+    const dim3 grid((Lq + attn_jvp::kBlockM - 1) / attn_jvp::kBlockM, H, B * eff_splits);
+    int rc;
+#define ATTN_JVP_DISPATCH(DD, SS)                                                                                  \
+    switch (mode) {                                                                                               \
+        case attn_jvp::kModeJvp: rc = launch<DD, attn_jvp::kModeJvp, SS>(maps, ka, grid, stream, dev); break;      \
+        case attn_jvp::kModeKvTangentFree:                                                                        \
+            rc = launch<DD, attn_jvp::kModeKvTangentFree, SS>(maps, ka, grid, stream, dev); break;                 \
+        default: rc = launch<DD, attn_jvp::kModeFwdOnly, SS>(maps, ka, grid, stream, dev); break;                  \
+    }
     if (D == 128) {
-        switch (mode) {
-            case attn_jvp::kModeJvp: return launch<128, attn_jvp::kModeJvp>(maps, ka, grid, stream, dev);
-            case attn_jvp::kModeKvTangentFree: return launch<128, attn_jvp::kModeKvTangentFree>(maps, ka, grid, stream, dev);
-            default: return launch<128, attn_jvp::kModeFwdOnly>(maps, ka, grid, stream, dev);
-        }
+        if (split) { ATTN_JVP_DISPATCH(128, true) } else { ATTN_JVP_DISPATCH(128, false) }
+    } else {
+        if (split) { ATTN_JVP_DISPATCH(64, true) } else { ATTN_JVP_DISPATCH(64, false) }
     }
-    switch (mode) {
-        case attn_jvp::kModeJvp: return launch<64, attn_jvp::kModeJvp>(maps, ka, grid, stream, dev);
-        case attn_jvp::kModeKvTangentFree: return launch<64, attn_jvp::kModeKvTangentFree>(maps, ka, grid, stream, dev);
-        default: return launch<64, attn_jvp::kModeFwdOnly>(maps, ka, grid, stream, dev);
-    }
+#undef ATTN_JVP_DISPATCH
+    if (rc != 0 || !split) return rc;
+
+    // merge the chunks (same stream: ordered after the partial kernel)
+    const long long n_threads = (long long)B * Lq * H * (D / 4);
+    const unsigned blocks = (unsigned)((n_threads + 255) / 256);
+    if (D == 128)
+        attn_jvp::attn_jvp_splitkv_merge_kernel<128><<<blocks, 256, 0, stream>>>(
+            ka.part_o, ka.part_to, ka.part_lse, ka.part_mu, ka.o, ka.to, lse, mu, B, H, Lq, eff_splits, fwd_only ? 0 : 1);
+    else
+        attn_jvp::attn_jvp_splitkv_merge_kernel<64><<<blocks, 256, 0, stream>>>(
+            ka.part_o, ka.part_to, ka.part_lse, ka.part_mu, ka.o, ka.to, lse, mu, B, H, Lq, eff_splits, fwd_only ? 0 : 1);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail("merge kernel launch", e);
+    return 0;
 }
 
 }  // namespace
@@ -199,13 +261,37 @@ extern "C" {
 
 int attn_jvp_fwd(const void* q, const void* k, const void* v, const void* tq, const void* tk, const void* tv,
                  void* o, void* to, float* lse, int B, int H, int Lq, int Lk, int D, float scale, unsigned flags) {
-    return run(q, k, v, tq, tk, tv, o, to, lse, B, H, Lq, Lk, D, scale, flags, tl_stream);
+    return run(q, k, v, tq, tk, tv, o, to, lse, nullptr, B, H, Lq, Lk, D, scale, flags, 1, nullptr, 0, tl_stream);
 }
 
 int attn_jvp_fwd_stream(const void* q, const void* k, const void* v, const void* tq, const void* tk, const void* tv,
                         void* o, void* to, float* lse, int B, int H, int Lq, int Lk, int D, float scale,
                         unsigned flags, void* cuda_stream) {
-    return run(q, k, v, tq, tk, tv, o, to, lse, B, H, Lq, Lk, D, scale, flags, static_cast<cudaStream_t>(cuda_stream));
+    return run(q, k, v, tq, tk, tv, o, to, lse, nullptr, B, H, Lq, Lk, D, scale, flags, 1, nullptr, 0,
+               static_cast<cudaStream_t>(cuda_stream));
+}
+
+int attn_jvp_fwd_mu(const void* q, const void* k, const void* v, const void* tq, const void* tk, const void* tv,
+                    void* o, void* to, float* lse, float* mu, int B, int H, int Lq, int Lk, int D, float scale,
+                    unsigned flags, void* cuda_stream) {
+    if (!mu) return ATTN_JVP_ERR_NULL;
+    return run(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, Lk, D, scale, flags, 1, nullptr, 0,
+               static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t attn_jvp_splitkv_workspace_bytes(int B, int H, int Lq, int Lk, int D, int splits) {
+    if (B < 1 || H < 1 || Lq < 1 || Lk < 1 || (D != 64 && D != 128) || splits < 1) return 0;
+    int tps = 0, eff = 1;
+    split_plan(Lk, splits, &tps, &eff);
+    if (eff <= 1) return 0;
+    return split_layout(B, H, Lq, D, eff).total;
+}
+
+int attn_jvp_fwd_splitkv(const void* q, const void* k, const void* v, const void* tq, const void* tk, const void* tv,
+                         void* o, void* to, float* lse, float* mu, int B, int H, int Lq, int Lk, int D, float scale,
+                         unsigned flags, int splits, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return run(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, Lk, D, scale, flags, splits, workspace, workspace_bytes,
+               static_cast<cudaStream_t>(cuda_stream));
 }
 
 int attn_jvp_set_stream(void* cuda_stream) {
@@ -243,6 +329,7 @@ const char* attn_jvp_strerror(int code) {
             return tl_strerror_buf;
         case ATTN_JVP_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired; the kernel stopped early";
         case ATTN_JVP_ERR_DEVICE_LAYOUT: return "the kernel's shared-memory layout did not fit; nothing was computed";
+        case ATTN_JVP_ERR_WORKSPACE: return "the split-KV workspace is smaller than attn_jvp_splitkv_workspace_bytes()";
         default: return "unknown error code";
     }
 }

@@ -79,9 +79,20 @@ struct KernelArgs {
     float* lse;
     int* host_status;   // mapped pinned host word, receives the timeout code
     int H, Lq, Lk;
-    int n_kv_tiles;
+    int n_kv_tiles;     // 64-key tiles in all of Lk
     float scale;        // s
     float scale_log2;   // s * log2(e)
+    // optional side output: mu = rowsum(P . tS) = d(LSE) along the tangent, fp32 [B][H][Lq] (may be null)
+    float* mu;
+    // split-KV mode: the keys are cut into `splits` chunks of `tiles_per_split` tiles; blockIdx.z = b * splits + s;
+    // chunk s writes normalised partial results (fp32) instead of the final outputs
+    int splits;
+    int tiles_per_split;
+    float* part_o;      // [splits][B][Lq][H][D]
+    float* part_to;     // [splits][B][Lq][H][D]
+    float* part_lse;    // [splits][B][H][Lq]
+    float* part_mu;     // [splits][B][H][Lq]
+    int B;
 };
 
 template <int D>
@@ -329,7 +340,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-template <int D, int MODE>
+template <int D, int MODE, bool kSplit>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_tq,
@@ -360,9 +371,11 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int lane = threadIdx.x & 31;
     const int q_tile = blockIdx.x;
     const int h = blockIdx.y;
-    const int b = blockIdx.z;
+    const int b = kSplit ? blockIdx.z / args.splits : blockIdx.z;
+    const int split = kSplit ? blockIdx.z % args.splits : 0;
+    const int tile0 = kSplit ? split * args.tiles_per_split : 0;       // first key tile of this CTA
     const int q0 = q_tile * kBlockM;
-    const int n_kv = args.n_kv_tiles;
+    const int n_kv = kSplit ? min(args.tiles_per_split, args.n_kv_tiles - tile0) : args.n_kv_tiles;
 #ifdef ATTN_JVP_TRACE
     const bool trace_on = blockIdx.x == gridDim.x / 2 && blockIdx.y == gridDim.y / 2 && blockIdx.z == 0;
 #endif
@@ -464,9 +477,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 // per 64-column half: [K_half (8 KB)][tK_half (8 KB)] so that [K ; tK] is one N = 128 operand
 #pragma unroll
                 for (int hf = 0; hf < kHalves; ++hf) {
-                    tma_load_4d(dst + hf * 2 * Plan::kKvHalfBytes, &tm_k, bar, hf * 64, h, j * kBlockN, b);
+                    tma_load_4d(dst + hf * 2 * Plan::kKvHalfBytes, &tm_k, bar, hf * 64, h, (tile0 + j) * kBlockN, b);
                     if (kHasTKV)
-                        tma_load_4d(dst + hf * 2 * Plan::kKvHalfBytes + Plan::kKvHalfBytes, &tm_tk, bar, hf * 64, h, j * kBlockN, b);
+                        tma_load_4d(dst + hf * 2 * Plan::kKvHalfBytes + Plan::kKvHalfBytes, &tm_tk, bar, hf * 64, h, (tile0 + j) * kBlockN, b);
                 }
                 return true;
             };
@@ -477,9 +490,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 // [V_half0][V_half1][tV_half0][tV_half1]: consecutive 64-wide N atoms of [V | tV]
 #pragma unroll
                 for (int hf = 0; hf < kHalves; ++hf) {
-                    tma_load_4d(dst + hf * Plan::kKvHalfBytes, &tm_v, bar, hf * 64, h, j * kBlockN, b);
+                    tma_load_4d(dst + hf * Plan::kKvHalfBytes, &tm_v, bar, hf * 64, h, (tile0 + j) * kBlockN, b);
                     if (kHasTKV)
-                        tma_load_4d(dst + (kHalves + hf) * Plan::kKvHalfBytes, &tm_tv, bar, hf * 64, h, j * kBlockN, b);
+                        tma_load_4d(dst + (kHalves + hf) * Plan::kKvHalfBytes, &tm_tv, bar, hf * 64, h, (tile0 + j) * kBlockN, b);
                 }
                 return true;
             };
@@ -720,7 +733,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             tc_wait_ld();
 
             // keys past Lk (zero-filled by TMA) must not enter the softmax
-            const int valid = args.Lk - j * kBlockN - half * kHalfN;    // valid columns of this half
+            const int valid = args.Lk - (tile0 + j) * kBlockN - half * kHalfN;    // valid columns of this half
             if (valid < kHalfN) {
                 const uint32_t masked = neg_scale ? 0x7F800000u : 0xFF800000u;   // -inf after scaling
 #pragma unroll
@@ -909,8 +922,12 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const float inv_l = 1.0f / l_tot;
             const float mu = r_tot * inv_l;
             const size_t row_off = ((static_cast<size_t>(b) * args.Lq + (in_range ? qi : 0)) * args.H + h) * D;
+            // split-KV: this chunk's normalised partial results go to the fp32 scratch of chunk `split`
+            const size_t part_off = kSplit ? static_cast<size_t>(split) * args.B * args.Lq * args.H * D + row_off : 0;
             __nv_bfloat16* o_row = args.o + row_off;
             __nv_bfloat16* to_row = kHasTQ ? args.to + row_off : nullptr;
+            float* po_row = kSplit ? args.part_o + part_off : nullptr;
+            float* pto_row = (kSplit && kHasTQ) ? args.part_to + part_off : nullptr;
 #pragma unroll 1
             for (int c0 = half * (D / kGroups); c0 < (half + 1) * (D / kGroups); c0 += 32) {
                 uint32_t ov[32];
@@ -918,29 +935,57 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 TMEM_LD32(tmem_o + lane_base + c0, ov, 0);
                 if (kHasTQ) TMEM_LD32(tmem_t + lane_base + c0, tvv, 0);
                 tc_wait_ld();
-                uint32_t po[16], pt[16];
+                if (kSplit) {
 #pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    const float o0 = __uint_as_float(ov[2 * c]) * inv_l;
-                    const float o1 = __uint_as_float(ov[2 * c + 1]) * inv_l;
-                    po[c] = pack_bf16(o0, o1);
-                    if (kHasTQ) {
-                        const float t0 = fmaf(-mu, o0, __uint_as_float(tvv[2 * c]) * inv_l);
-                        const float t1 = fmaf(-mu, o1, __uint_as_float(tvv[2 * c + 1]) * inv_l);
-                        pt[c] = pack_bf16(t0, t1);
+                    for (int c = 0; c < 32; ++c) {
+                        const float o0 = __uint_as_float(ov[c]) * inv_l;
+                        ov[c] = __float_as_uint(o0);
+                        if (kHasTQ) tvv[c] = __float_as_uint(fmaf(-mu, o0, __uint_as_float(tvv[c]) * inv_l));
                     }
-                }
-                if (in_range) {
+                    if (in_range) {
 #pragma unroll
-                    for (int v4 = 0; v4 < 4; ++v4) {
-                        *reinterpret_cast<uint4*>(o_row + c0 + v4 * 8) = make_uint4(po[4 * v4], po[4 * v4 + 1], po[4 * v4 + 2], po[4 * v4 + 3]);
-                        if (kHasTQ)
-                            *reinterpret_cast<uint4*>(to_row + c0 + v4 * 8) = make_uint4(pt[4 * v4], pt[4 * v4 + 1], pt[4 * v4 + 2], pt[4 * v4 + 3]);
+                        for (int v4 = 0; v4 < 8; ++v4) {
+                            *reinterpret_cast<uint4*>(po_row + c0 + v4 * 4) = make_uint4(ov[4 * v4], ov[4 * v4 + 1], ov[4 * v4 + 2], ov[4 * v4 + 3]);
+                            if (kHasTQ)
+                                *reinterpret_cast<uint4*>(pto_row + c0 + v4 * 4) = make_uint4(tvv[4 * v4], tvv[4 * v4 + 1], tvv[4 * v4 + 2], tvv[4 * v4 + 3]);
+                        }
+                    }
+                } else {
+                    uint32_t po[16], pt[16];
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        const float o0 = __uint_as_float(ov[2 * c]) * inv_l;
+                        const float o1 = __uint_as_float(ov[2 * c + 1]) * inv_l;
+                        po[c] = pack_bf16(o0, o1);
+                        if (kHasTQ) {
+                            const float t0 = fmaf(-mu, o0, __uint_as_float(tvv[2 * c]) * inv_l);
+                            const float t1 = fmaf(-mu, o1, __uint_as_float(tvv[2 * c + 1]) * inv_l);
+                            pt[c] = pack_bf16(t0, t1);
+                        }
+                    }
+                    if (in_range) {
+#pragma unroll
+                        for (int v4 = 0; v4 < 4; ++v4) {
+                            *reinterpret_cast<uint4*>(o_row + c0 + v4 * 8) = make_uint4(po[4 * v4], po[4 * v4 + 1], po[4 * v4 + 2], po[4 * v4 + 3]);
+                            if (kHasTQ)
+                                *reinterpret_cast<uint4*>(to_row + c0 + v4 * 8) = make_uint4(pt[4 * v4], pt[4 * v4 + 1], pt[4 * v4 + 2], pt[4 * v4 + 3]);
+                        }
                     }
                 }
             }
             if (in_range && half == 0) {
-                args.lse[(static_cast<size_t>(b) * args.H + h) * args.Lq + qi] = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
+                // L = m + log l (natural log); mu = r / l, plus the constant that was taken out of tS
+                const float lse_val = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
+                const float mu_val = kHasTQ ? mu + ts_shift : 0.0f;
+                const size_t idx = (static_cast<size_t>(b) * args.H + h) * args.Lq + qi;
+                if (kSplit) {
+                    const size_t pidx = static_cast<size_t>(split) * args.B * args.H * args.Lq + idx;
+                    args.part_lse[pidx] = lse_val;
+                    args.part_mu[pidx] = mu_val;
+                } else {
+                    args.lse[idx] = lse_val;
+                    if (args.mu != nullptr) args.mu[idx] = mu_val;
+                }
             }
         }
     }
@@ -954,6 +999,72 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     if (warp == kMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Split-KV merge.  Chunk c of the keys gave (O_c, tO_c, LSE_c, mu_c), each normalised within the chunk.
+// With w_c = exp(LSE_c - LSE), LSE = log sum_c exp(LSE_c):
+//     O = sum_c w_c O_c,   mu = sum_c w_c mu_c,   tO = sum_c w_c (tO_c + mu_c O_c) - mu O
+// (the aggregated form of Appendix C.1 regrouped by chunk; mu = rowsum(P . tS) = d LSE).
+// One thread per (row, 4 columns).
+// ---------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256)
+attn_jvp_splitkv_merge_kernel(const float* __restrict__ part_o, const float* __restrict__ part_to,
+                              const float* __restrict__ part_lse, const float* __restrict__ part_mu,
+                              __nv_bfloat16* __restrict__ o, __nv_bfloat16* __restrict__ to,
+                              float* __restrict__ lse, float* __restrict__ mu,
+                              int B, int H, int Lq, int splits, int has_tangent) {
+    constexpr int kVecPerRow = D / 4;
+    const long long n_rows = static_cast<long long>(B) * Lq * H;
+    const long long gid = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const long long r = gid / kVecPerRow;             // row index in [B][Lq][H] order
+    const int v = static_cast<int>(gid % kVecPerRow);
+    if (r >= n_rows) return;
+    const int h = static_cast<int>(r % H);
+    const long long bl = r / H;
+    const int l = static_cast<int>(bl % Lq);
+    const int b = static_cast<int>(bl / Lq);
+    const size_t stat = (static_cast<size_t>(b) * H + h) * Lq + l;         // index in [B][H][Lq]
+    const size_t stat_stride = static_cast<size_t>(B) * H * Lq;
+    const size_t vec_stride = static_cast<size_t>(n_rows) * D;
+
+    float lse_max = -INFINITY;
+    for (int c = 0; c < splits; ++c) lse_max = fmaxf(lse_max, part_lse[c * stat_stride + stat]);
+    float denom = 0.0f;
+    for (int c = 0; c < splits; ++c) denom += __expf(part_lse[c * stat_stride + stat] - lse_max);
+    const float inv_denom = 1.0f / denom;
+
+    float4 acc_o = make_float4(0.f, 0.f, 0.f, 0.f), acc_t = make_float4(0.f, 0.f, 0.f, 0.f);
+    float mu_tot = 0.0f;
+    for (int c = 0; c < splits; ++c) {
+        const float w = __expf(part_lse[c * stat_stride + stat] - lse_max) * inv_denom;
+        const float4 oc = *reinterpret_cast<const float4*>(part_o + c * vec_stride + static_cast<size_t>(r) * D + v * 4);
+        acc_o.x = fmaf(w, oc.x, acc_o.x); acc_o.y = fmaf(w, oc.y, acc_o.y);
+        acc_o.z = fmaf(w, oc.z, acc_o.z); acc_o.w = fmaf(w, oc.w, acc_o.w);
+        if (has_tangent) {
+            const float mc = part_mu[c * stat_stride + stat];
+            const float4 tc = *reinterpret_cast<const float4*>(part_to + c * vec_stride + static_cast<size_t>(r) * D + v * 4);
+            mu_tot = fmaf(w, mc, mu_tot);
+            acc_t.x = fmaf(w, fmaf(mc, oc.x, tc.x), acc_t.x); acc_t.y = fmaf(w, fmaf(mc, oc.y, tc.y), acc_t.y);
+            acc_t.z = fmaf(w, fmaf(mc, oc.z, tc.z), acc_t.z); acc_t.w = fmaf(w, fmaf(mc, oc.w, tc.w), acc_t.w);
+        }
+    }
+    const size_t out = static_cast<size_t>(r) * D + v * 4;
+    uint2 po;
+    po.x = pack_bf16(acc_o.x, acc_o.y);
+    po.y = pack_bf16(acc_o.z, acc_o.w);
+    *reinterpret_cast<uint2*>(o + out) = po;
+    if (has_tangent) {
+        uint2 pt;
+        pt.x = pack_bf16(fmaf(-mu_tot, acc_o.x, acc_t.x), fmaf(-mu_tot, acc_o.y, acc_t.y));
+        pt.y = pack_bf16(fmaf(-mu_tot, acc_o.z, acc_t.z), fmaf(-mu_tot, acc_o.w, acc_t.w));
+        *reinterpret_cast<uint2*>(to + out) = pt;
+    }
+    if (v == 0) {
+        lse[stat] = lse_max + __logf(denom);
+        if (mu != nullptr) mu[stat] = has_tangent ? mu_tot : 0.0f;
     }
 }
 
