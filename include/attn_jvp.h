@@ -61,6 +61,10 @@ extern "C" {
 #define ATTN_JVP_ERR_DEVICE_TIMEOUT 10  /* a bounded device-side wait expired */
 #define ATTN_JVP_ERR_DEVICE_LAYOUT  11  /* the kernel's shared-memory layout did not fit (reported like a timeout) */
 #define ATTN_JVP_ERR_WORKSPACE      12  /* split-KV workspace too small */
+#define ATTN_JVP_ERR_STATIC_SCRATCH 13  /* the call needs more scratch than ATTN_JVP_STATIC_SCRATCH_BYTES */
+
+/* Size of the scratch buffer built into the library for attn_jvp_fwd_splitkv_static (32 MiB). */
+#define ATTN_JVP_STATIC_SCRATCH_BYTES (32u * 1024u * 1024u)
 
 /*
  * attn_jvp_fwd -- O, tO and LSE of Algorithm 2 in one pass, on the stream set
@@ -119,6 +123,41 @@ int attn_jvp_fwd_splitkv(const void* q, const void* k, const void* v,
                          int B, int H, int Lq, int Lk, int D,
                          float scale, unsigned flags, int splits,
                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * attn_jvp_fwd_splitkv_static -- the split-KV computation of attn_jvp_fwd_splitkv for callers that are not
+ * allowed to allocate GPU memory.  (No counterpart in the paper: this is a packaging variant, the arithmetic
+ * is that of attn_jvp_fwd_splitkv.)
+ *
+ * Who needs it: code that runs where a cudaMalloc is off limits -- inside a region being captured into a CUDA
+ * graph or replayed from one, in a real-time or serving loop whose memory was fixed at start-up, under a
+ * framework whose allocator must own every byte, or in a process whose memory budget is already spent.  Such
+ * a caller cannot provide the workspace that attn_jvp_fwd_splitkv asks for, so this entry point brings its own:
+ * a fixed array of ATTN_JVP_STATIC_SCRATCH_BYTES (32 MiB) that is part of the library's device image.  Every GPU
+ * on which the library is loaded gives up that much memory until the process exits, whether or not this
+ * function is ever called.
+ *
+ * Behaviour
+ *   - Arguments as attn_jvp_fwd_splitkv, without workspace / workspace_bytes.  Inputs and outputs are still the
+ *     caller's device buffers.
+ *   - The function itself calls no cudaMalloc / cudaFree / cudaHostAlloc and no allocating library routine.
+ *     (It also skips the pinned status word the other entry points create on first use; a device-side timeout in
+ *     a call made before any other entry point ran on this device is then only visible as later launches
+ *     returning at once.)
+ *   - A call whose chunks need more than ATTN_JVP_STATIC_SCRATCH_BYTES (see attn_jvp_splitkv_workspace_bytes)
+ *     is refused with ATTN_JVP_ERR_STATIC_SCRATCH and nothing is enqueued; attn_jvp_strerror gives both sizes.
+ *   - The first call on each device looks up the array's device address (with that device current).  Make that
+ *     first call outside of any stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the previous call left in it.  Nothing in
+ *     it has to start at zero: every value that the merge step reads is written by the same call first.  Two calls
+ *     that overlap on the GPU (different streams, no dependency between them) race on the array and produce
+ *     garbage; calls on one stream, or otherwise ordered, are fine.
+ */
+int attn_jvp_fwd_splitkv_static(const void* q, const void* k, const void* v,
+                                const void* tq, const void* tk, const void* tv,
+                                void* o, void* to, float* lse, float* mu,
+                                int B, int H, int Lq, int Lk, int D,
+                                float scale, unsigned flags, int splits, void* cuda_stream);
 
 /* Sets the stream attn_jvp_fwd launches on for the calling host thread
  * (thread-local; NULL = legacy default stream).  Always returns 0. */

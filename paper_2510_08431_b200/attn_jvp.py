@@ -18,9 +18,11 @@ FWD_ONLY = 0x2
 
 ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED_D, ERR_ALIGN, ERR_FLAGS = 1, 2, 3, 4, 5
 ERR_SCALE, ERR_ALIAS, ERR_ARCH, ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_DEVICE_LAYOUT, ERR_WORKSPACE = 6, 7, 8, 9, 10, 11, 12
+ERR_STATIC_SCRATCH = 13
+STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 EXPORTS = ("attn_jvp_fwd", "attn_jvp_fwd_stream", "attn_jvp_fwd_mu", "attn_jvp_splitkv_workspace_bytes",
-           "attn_jvp_fwd_splitkv", "attn_jvp_set_stream", "attn_jvp_device_status", "attn_jvp_strerror",
+           "attn_jvp_fwd_splitkv", "attn_jvp_fwd_splitkv_static", "attn_jvp_set_stream", "attn_jvp_device_status", "attn_jvp_strerror",
            "attn_jvp_version")
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libattn_jvp.so")
@@ -60,6 +62,8 @@ def load():
             lib.attn_jvp_splitkv_workspace_bytes.restype = ctypes.c_size_t
             lib.attn_jvp_fwd_splitkv.argtypes = [vp] * 10 + [ci] * 5 + [cf, cu, ci, vp, ctypes.c_size_t, vp]
             lib.attn_jvp_fwd_splitkv.restype = ci
+            lib.attn_jvp_fwd_splitkv_static.argtypes = [vp] * 10 + [ci] * 5 + [cf, cu, ci, vp]
+            lib.attn_jvp_fwd_splitkv_static.restype = ci
             lib.attn_jvp_set_stream.argtypes = [vp]
             lib.attn_jvp_set_stream.restype = ci
             lib.attn_jvp_device_status.argtypes = []
@@ -123,6 +127,17 @@ def attn_jvp_fwd_splitkv(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, Lk, D, s
     return int(load().attn_jvp_fwd_splitkv(_ptr(q), _ptr(k), _ptr(v), _ptr(tq), _ptr(tk), _ptr(tv), _ptr(o),
                                            _ptr(to), _ptr(lse), _ptr(mu), B, H, Lq, Lk, D, float(scale), int(flags),
                                            int(splits), _ptr(workspace), int(workspace_bytes), _ptr(cuda_stream)))
+
+
+def attn_jvp_fwd_splitkv_static(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, Lk, D, scale, flags, splits,
+                                cuda_stream) -> int:
+    """Split-KV for callers that may not allocate GPU memory (inside CUDA-graph capture, fixed-memory serving
+    loops, allocator-owned processes): the chunk partials go to a 32 MiB buffer built into the library instead of
+    a caller-provided workspace.  Calls larger than that are refused (ERR_STATIC_SCRATCH); calls that overlap on
+    the GPU race on the shared buffer.  Raw call: tensors or device addresses in, return code out."""
+    return int(load().attn_jvp_fwd_splitkv_static(_ptr(q), _ptr(k), _ptr(v), _ptr(tq), _ptr(tk), _ptr(tv), _ptr(o),
+                                                  _ptr(to), _ptr(lse), _ptr(mu), B, H, Lq, Lk, D, float(scale),
+                                                  int(flags), int(splits), _ptr(cuda_stream)))
 
 
 def _check(t, name, shape):

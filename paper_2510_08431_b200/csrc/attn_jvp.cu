@@ -127,7 +127,7 @@ void split_plan(int Lk, int splits, int* tiles_per_split, int* eff_splits) {
 
 int run(const void* q, const void* k, const void* v, const void* tq, const void* tk, const void* tv,
         void* o, void* to, float* lse, float* mu, int B, int H, int Lq, int Lk, int D, float scale, unsigned flags,
-        int splits, void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+        int splits, void* workspace, size_t workspace_bytes, cudaStream_t stream, bool may_allocate = true) {
     // ---- validation: nothing is enqueued unless everything checks out ----
     if (flags & ~(ATTN_JVP_KV_TANGENT_FREE | ATTN_JVP_FWD_ONLY)) return ATTN_JVP_ERR_FLAGS;
     const bool fwd_only = (flags & ATTN_JVP_FWD_ONLY) != 0;
@@ -179,7 +179,7 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     if (major != 10) return ATTN_JVP_ERR_ARCH;
 
     if (int rc = get_encode_fn()) return rc;
-    if (!g_host_status[dev]) {
+    if (!g_host_status[dev] && may_allocate) {
         int* hp = nullptr;
         e = cudaHostAlloc((void**)&hp, sizeof(int), cudaHostAllocMapped);
         if (e != cudaSuccess) return cuda_fail("cudaHostAlloc(status word)", e);
@@ -204,7 +204,7 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     ka.o = reinterpret_cast<__nv_bfloat16*>(o);
     ka.to = reinterpret_cast<__nv_bfloat16*>(to);
     ka.lse = lse;
-    ka.host_status = g_host_status_dev[dev];
+    ka.host_status = g_host_status_dev[dev];   // null if no call on this device was allowed to allocate it yet
     ka.H = H;
     ka.Lq = Lq;
     ka.Lk = Lk;
@@ -294,6 +294,38 @@ int attn_jvp_fwd_splitkv(const void* q, const void* k, const void* v, const void
                static_cast<cudaStream_t>(cuda_stream));
 }
 
+// Scratch for callers that cannot allocate: lives in the library's device image, so every GPU that loads
+// the library holds these bytes until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[ATTN_JVP_STATIC_SCRATCH_BYTES];
+static void* g_static_scratch_dev[kMaxDevices] = {};   // device address of the array, looked up once per device
+
+int attn_jvp_fwd_splitkv_static(const void* q, const void* k, const void* v, const void* tq, const void* tk,
+                                const void* tv, void* o, void* to, float* lse, float* mu, int B, int H, int Lq, int Lk,
+                                int D, float scale, unsigned flags, int splits, void* cuda_stream) {
+    if (B < 1 || H < 1 || Lq < 1 || Lk < 1 || splits < 1) return ATTN_JVP_ERR_SHAPE;
+    if (D != 64 && D != 128) return ATTN_JVP_ERR_UNSUPPORTED_D;
+    const size_t need = attn_jvp_splitkv_workspace_bytes(B, H, Lq, Lk, D, splits);
+    if (need > (size_t)ATTN_JVP_STATIC_SCRATCH_BYTES) {
+        snprintf(tl_cuda_msg, sizeof tl_cuda_msg, "this call needs %zu bytes of scratch, the built-in buffer holds %zu",
+                 need, (size_t)ATTN_JVP_STATIC_SCRATCH_BYTES);
+        return ATTN_JVP_ERR_STATIC_SCRATCH;
+    }
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail("cudaGetDevice", e);
+    if (dev < 0 || dev >= kMaxDevices) return ATTN_JVP_ERR_ARCH;
+    if (!g_static_scratch_dev[dev]) {
+        // In host code the array's name only stands for the symbol; its address on the current device has to be
+        // asked for.  Done once per device, on the first call (which should therefore precede any stream capture).
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess) return cuda_fail("cudaGetSymbolAddress(static scratch)", e);
+        g_static_scratch_dev[dev] = p;
+    }
+    return run(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, Lk, D, scale, flags, splits, g_static_scratch_dev[dev],
+               (size_t)ATTN_JVP_STATIC_SCRATCH_BYTES, static_cast<cudaStream_t>(cuda_stream), /*may_allocate=*/false);
+}
+
 int attn_jvp_set_stream(void* cuda_stream) {
     tl_stream = static_cast<cudaStream_t>(cuda_stream);
     return 0;
@@ -330,6 +362,9 @@ const char* attn_jvp_strerror(int code) {
         case ATTN_JVP_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired; the kernel stopped early";
         case ATTN_JVP_ERR_DEVICE_LAYOUT: return "the kernel's shared-memory layout did not fit; nothing was computed";
         case ATTN_JVP_ERR_WORKSPACE: return "the split-KV workspace is smaller than attn_jvp_splitkv_workspace_bytes()";
+        case ATTN_JVP_ERR_STATIC_SCRATCH:
+            snprintf(tl_strerror_buf, sizeof tl_strerror_buf, "built-in scratch too small: %s", tl_cuda_msg);
+            return tl_strerror_buf;
         default: return "unknown error code";
     }
 }

@@ -43,7 +43,7 @@ def test_every_declared_symbol_is_exported(lib):
 def test_version_and_strerror(lib):
     assert lib.attn_jvp_version() >= 100
     assert lib.attn_jvp_strerror(0) == "ok"
-    for code in range(1, 13):
+    for code in range(1, 14):
         assert lib.attn_jvp_strerror(code) not in ("ok", "unknown error code")
     assert lib.attn_jvp_strerror(99) == "unknown error code"
 
