@@ -185,6 +185,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--splits", type=int, default=1, help="key chunks (split-KV entry point) for few-query workloads")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = synth.WORKLOADS[args.workload]
@@ -223,10 +224,14 @@ def main():
     if algorithmic_bytes(w) <= 2 * 126e6:
         flush = torch.empty(512 * 1024 * 1024, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
+    workspace = None
+    if args.splits > 1:
+        need = aj.attn_jvp_splitkv_workspace_bytes(w.B, w.H, w.Lq, w.Lk, w.D, args.splits)
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
 
     def step(fwd_only=False):
         aj.attention_jvp(g["q"], g["k"], g["v"], g["tq"], g["tk"], g["tv"], scale=w.scale, fwd_only=fwd_only,
-                         out=(o, None if fwd_only else to, lse))
+                         out=(o, None if fwd_only else to, lse), splits=args.splits, workspace=workspace)
 
     def timed(n_steps, fwd_only=False):
         """Per-launch CUDA-event durations (ms) on the launching stream."""
@@ -326,7 +331,8 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": workload_config(w), "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps,
+                "config": workload_config(w, extra={"splits": args.splits} if args.splits > 1 else None),
+                "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * (2 if args.splits > 1 else 1),
                 "roofline": roofline,
                 "jvp_over_fwd": (kernel_ms / fwd_ms) if fwd_ms else None, "fwd_only_ms": fwd_ms,
                 "per_launch_ms": {"median": statistics.median(per_launch), "best": min(per_launch)}}

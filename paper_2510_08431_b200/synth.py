@@ -55,6 +55,9 @@ WORKLOADS = {
     "video_dit_14b": Workload("video_dit_14b", 1, 40, 32760, 32760, 128, 1.0, 0.5, 3),
     "cross_attn_14b": Workload("cross_attn_14b", 1, 40, 32760, 512, 128, 1.0, 1.0, 4,
                                kv_tangent_free=True),
+    # not one of the five benchmark configs: few queries against a long key sequence, the case the
+    # split-KV entry point exists for (32 query tiles x heads CTAs would fill a fifth of the GPU)
+    "few_q_long_k": Workload("few_q_long_k", 1, 8, 512, 32760, 128, 1.0, 0.5, 5),
 }
 
 
