@@ -31,7 +31,7 @@ if ROOT not in sys.path:
 import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
-from paper_2510_08431_b200 import synth  # noqa: E402
+from paper_2510_08431_b200 import replicas, synth  # noqa: E402
 
 METRIC = "attention-JVP TFLOP/s (12*B*H*Lq*Lk*D)"
 UNIT = "TFLOP/s"
@@ -264,12 +264,8 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     kernel_ms = sum(per_launch) / len(per_launch)
     total_ms = t_begin.elapsed_time(t_end) if flush is None else sum(per_launch)
-    tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-    total_ms = float(tt.item())
-    ms_per_step = total_ms / args.steps
-    value = world * w.flops / (ms_per_step * 1e-3) / 1e12
+    flops_per_s, ms_per_step, _ = replicas.aggregate_throughput(w.flops, total_ms, args.steps, dist, dev)
+    value = flops_per_s / 1e12
 
     # forward-only of the same kernel, for the JVP / forward cost ratio
     fwd_ms = None
@@ -303,10 +299,7 @@ def main():
             e2e_step()
         b.record(stream)
         barrier()
-        et = torch.tensor([a.elapsed_time(b)], dtype=torch.float64, device=dev)
-        if dist is not None:
-            dist.all_reduce(et, op=dist.ReduceOp.MAX)
-        e2e_ms = float(et.item()) / n_e2e
+        e2e_ms = replicas.max_over_ranks(a.elapsed_time(b), dist, dev) / n_e2e
         e2e = {"value": world * w.flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": n_e2e}
     st = aj.attn_jvp_device_status()

@@ -99,7 +99,7 @@ def test_single_key_returns_v_and_tv(aj):
 
 def _rel_l2_only(oracle, x, B, H, Lq, Lk, D, scale, o, to, lse):
     """For O(1)-magnitude, strongly peaked cases: the max-norm gate is sized for the benchmark workloads
-    (outputs far below 1) and bf16 rounding of H~ can legitimately exceed it, so judge on relative L2."""
+    (outputs far below 1) and bf16 rounding of H~ can legitimately exceed it, so the check is on relative L2."""
     rows = np.arange(B * H * Lq)
     rO, rtO, rL, _ = U.oracle_rows(oracle, x, B, H, Lq, Lk, D, scale, rows)
     for name, got, ref in (("O", U.rows_of(o, rows, D), rO), ("tO", U.rows_of(to, rows, D), rtO)):
