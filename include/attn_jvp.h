@@ -168,9 +168,19 @@ int attn_jvp_set_stream(void* cuda_stream);
  * function: 0, or ATTN_JVP_ERR_DEVICE_TIMEOUT if a bounded wait inside a
  * kernel expired (ATTN_JVP_ERR_DEVICE_LAYOUT if its shared-memory layout did
  * not fit).  Meaningful once the caller has synchronised the stream(s) the
- * kernels ran on; reading it clears it.  Does not synchronise.
+ * kernels ran on; reading it clears it (and lets later launches run again).
+ * Copies one word from the device, so it orders itself after work on the
+ * legacy default stream; it does not wait for other streams.
  */
 int attn_jvp_device_status(void);
+
+/*
+ * Self-test of the failure path (no counterpart in the paper): enqueues a one-warp kernel that waits on a
+ * barrier nothing ever signals.  The wait expires after its time limit (about 2 s), the kernel ends normally,
+ * and attn_jvp_device_status() then reports ATTN_JVP_ERR_DEVICE_TIMEOUT, exactly as it would for a stalled
+ * attention kernel.  Nothing is trapped or faulted; the device stays usable.  Returns 0 when enqueued.
+ */
+int attn_jvp_selftest_bounded_wait(void* cuda_stream);
 
 /* Human-readable text for a return code; for ATTN_JVP_ERR_CUDA the text of the
  * last failing CUDA call on this thread is appended.  Never NULL. */

@@ -22,7 +22,7 @@ ERR_STATIC_SCRATCH = 13
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 EXPORTS = ("attn_jvp_fwd", "attn_jvp_fwd_stream", "attn_jvp_fwd_mu", "attn_jvp_splitkv_workspace_bytes",
-           "attn_jvp_fwd_splitkv", "attn_jvp_fwd_splitkv_static", "attn_jvp_set_stream", "attn_jvp_device_status", "attn_jvp_strerror",
+           "attn_jvp_fwd_splitkv", "attn_jvp_fwd_splitkv_static", "attn_jvp_selftest_bounded_wait", "attn_jvp_set_stream", "attn_jvp_device_status", "attn_jvp_strerror",
            "attn_jvp_version")
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libattn_jvp.so")
@@ -64,6 +64,8 @@ def load():
             lib.attn_jvp_fwd_splitkv.restype = ci
             lib.attn_jvp_fwd_splitkv_static.argtypes = [vp] * 10 + [ci] * 5 + [cf, cu, ci, vp]
             lib.attn_jvp_fwd_splitkv_static.restype = ci
+            lib.attn_jvp_selftest_bounded_wait.argtypes = [vp]
+            lib.attn_jvp_selftest_bounded_wait.restype = ci
             lib.attn_jvp_set_stream.argtypes = [vp]
             lib.attn_jvp_set_stream.restype = ci
             lib.attn_jvp_device_status.argtypes = []
@@ -94,6 +96,11 @@ def attn_jvp_version() -> int:
 
 def attn_jvp_set_stream(cuda_stream) -> int:
     return int(load().attn_jvp_set_stream(_ptr(cuda_stream)))
+
+
+def attn_jvp_selftest_bounded_wait(cuda_stream=None) -> int:
+    """Enqueues the bounded-wait self-test kernel (its wait expires after about 2 s); see include/attn_jvp.h."""
+    return int(load().attn_jvp_selftest_bounded_wait(_ptr(cuda_stream)))
 
 
 def attn_jvp_device_status() -> int:

@@ -326,6 +326,21 @@ int attn_jvp_fwd_splitkv_static(const void* q, const void* k, const void* v, con
                (size_t)ATTN_JVP_STATIC_SCRATCH_BYTES, static_cast<cudaStream_t>(cuda_stream), /*may_allocate=*/false);
 }
 
+int attn_jvp_selftest_bounded_wait(void* cuda_stream) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail("cudaGetDevice", e);
+    if (dev < 0 || dev >= kMaxDevices) return ATTN_JVP_ERR_ARCH;
+    int major = 0;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) return cuda_fail("cudaDeviceGetAttribute", e);
+    if (major != 10) return ATTN_JVP_ERR_ARCH;
+    attn_jvp::bounded_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(g_host_status_dev[dev]);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail("self-test kernel launch", e);
+    return 0;
+}
+
 int attn_jvp_set_stream(void* cuda_stream) {
     tl_stream = static_cast<cudaStream_t>(cuda_stream);
     return 0;
@@ -334,11 +349,17 @@ int attn_jvp_set_stream(void* cuda_stream) {
 int attn_jvp_device_status(void) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    int st = 0;
     int* hp = g_host_status[dev];
-    if (!hp) return 0;
-    const int st = *reinterpret_cast<volatile int*>(hp);
-    if (st != 0) {
-        *reinterpret_cast<volatile int*>(hp) = 0;
+    if (hp) {
+        st = *reinterpret_cast<volatile int*>(hp);
+        if (st != 0) *reinterpret_cast<volatile int*>(hp) = 0;
+    }
+    // The kernels also raise a device-side flag (later launches test it and return at once).  It is the only
+    // record when no status word exists yet, i.e. when only the allocation-free entry point has run here.
+    int flag = 0;
+    if (cudaMemcpyFromSymbol(&flag, attn_jvp::g_abort_flag, sizeof(int)) == cudaSuccess && flag != 0) {
+        if (st == 0) st = ATTN_JVP_ERR_DEVICE_TIMEOUT;
         const int zero = 0;
         cudaMemcpyToSymbol(attn_jvp::g_abort_flag, &zero, sizeof(int));   // let later launches run again
     }

@@ -1003,6 +1003,24 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 }
 
 // ---------------------------------------------------------------------------------------------
+// Self-test of the bounded wait: one warp waits on a barrier on which nothing ever arrives.  The wait
+// must give up after its time limit, record ATTN_JVP_ERR_DEVICE_TIMEOUT and let the kernel end normally
+// (no trap, no endless loop), leaving the context usable.
+// ---------------------------------------------------------------------------------------------
+__global__ void bounded_wait_selftest_kernel(int* host_status) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int cta_abort;
+    if (threadIdx.x == 0) {
+        cta_abort = 0;
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    AbortState st{&cta_abort, host_status};
+    (void)mbar_wait_warp(smem_u32(&bar), 0, st);
+}
+
+// ---------------------------------------------------------------------------------------------
 // Split-KV merge.  Chunk c of the keys gave (O_c, tO_c, LSE_c, mu_c), each normalised within the chunk.
 // With w_c = exp(LSE_c - LSE), LSE = log sum_c exp(LSE_c):
 //     O = sum_c w_c O_c,   mu = sum_c w_c mu_c,   tO = sum_c w_c (tO_c + mu_c O_c) - mu O
