@@ -175,6 +175,21 @@ int attn_jvp_set_stream(void* cuda_stream);
 int attn_jvp_device_status(void);
 
 /*
+ * attn_jvp_qknorm_fwd -- RMS normalisation over the head dimension together with its forward-mode tangent,
+ * the step that produces q, k, tq, tk for the attention kernel in a DiT block with QK normalisation (Sec. 3.1;
+ * Appendix C.2 restructures an RMSNorm layer for JVP mode).  Per row x in R^D, with frozen weight w:
+ *     n = sqrt(mean(x^2) + eps),   y = w . x / n,   ty = w . (tx / n - x (x . tx) / (D n^3)).
+ *
+ *   x, tx   device, bf16, `rows` rows of D contiguous elements (any [..][D] layout, e.g. [B][L][H][D]);
+ *           tx may be NULL together with ty (primal only).
+ *   w       device, fp32 [D].      y, ty   device, bf16, same shape as x.
+ *   rows >= 1; D is 64 or 128; eps >= 0; all pointers 16-byte aligned; outputs must not overlap inputs.
+ * Asynchronous on `cuda_stream`; returns 0 or an ATTN_JVP_ERR_* code (nothing enqueued on error).
+ */
+int attn_jvp_qknorm_fwd(const void* x, const void* tx, const float* w, void* y, void* ty,
+                        long long rows, int D, float eps, void* cuda_stream);
+
+/*
  * Self-test of the failure path (no counterpart in the paper): enqueues a one-warp kernel that waits on a
  * barrier nothing ever signals.  The wait expires after its time limit (about 2 s), the kernel ends normally,
  * and attn_jvp_device_status() then reports ATTN_JVP_ERR_DEVICE_TIMEOUT, exactly as it would for a stalled

@@ -317,3 +317,33 @@ int attn_jvp_oracle_threads(void)
     return 1;
 #endif
 }
+
+/* ------------------------------------------------------------------------- */
+/*
+ * RMS normalisation over the last dimension and its forward-mode tangent (the QK normalisation of the DiT
+ * attention block, Sec. 3.1, in the JVP-mode layer form of Appendix C.2), written out from the definition:
+ *     n = sqrt(mean_d x_d^2 + eps),  y_d = w_d x_d / n,
+ *     ty_d = d/d(eps') y_d(x + eps' tx) at 0 = w_d (tx_d / n - x_d (sum_e x_e tx_e) / (D n^3)).
+ * x, tx, y, ty: [rows][D] doubles; w: [D].  tx / ty may be NULL.
+ */
+int rmsnorm_jvp_f64(const double *x, const double *tx, const double *w, long rows, long D, double eps,
+                    double *y, double *ty)
+{
+    if (rows < 1 || D < 1) return 1;
+    for (long r = 0; r < rows; ++r) {
+        const double *xr = x + r * D;
+        double ss = 0.0;
+        for (long d = 0; d < D; ++d) ss += xr[d] * xr[d];
+        const double n = sqrt(ss / (double)D + eps);
+        for (long d = 0; d < D; ++d) y[r * D + d] = w[d] * xr[d] / n;
+        if (tx && ty) {
+            const double *tr = tx + r * D;
+            double dot = 0.0;
+            for (long d = 0; d < D; ++d) dot += xr[d] * tr[d];
+            /* dn = dot / (D n) ; d(x/n) = tx/n - x dn / n^2 */
+            const double dn = dot / ((double)D * n);
+            for (long d = 0; d < D; ++d) ty[r * D + d] = w[d] * (tr[d] / n - xr[d] * dn / (n * n));
+        }
+    }
+    return 0;
+}

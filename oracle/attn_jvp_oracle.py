@@ -172,3 +172,23 @@ def splitkv_merge(O_c, tO_c, LSE_c, MU_c):
     mu = sum(w[c] * MU_c[c] for c in range(len(O_c)))
     tO = sum(w[c][:, None] * (tO_c[c] + MU_c[c][:, None] * O_c[c]) for c in range(len(O_c))) - mu[:, None] * O
     return O, tO, LSE, mu
+
+
+def rmsnorm_jvp(x, tx, w, eps):
+    """RMS normalisation over the last axis and its tangent (fp64).  x, tx: [rows][D]; w: [D].  Returns (y, ty)."""
+    lib = _load()
+    if not hasattr(lib, "_rms_ready"):
+        dp = ctypes.POINTER(ctypes.c_double)
+        lib.rmsnorm_jvp_f64.argtypes = [dp, dp, dp, ctypes.c_long, ctypes.c_long, ctypes.c_double, dp, dp]
+        lib.rmsnorm_jvp_f64.restype = ctypes.c_int
+        lib._rms_ready = True
+    x = _f64(x)
+    rows, D = x.shape
+    tx = _f64(tx, (rows, D))
+    w = _f64(w, (D,))
+    y = np.empty((rows, D))
+    ty = None if tx is None else np.empty((rows, D))
+    rc = lib.rmsnorm_jvp_f64(_dptr(x), _dptr(tx), _dptr(w), rows, D, float(eps), _dptr(y), _dptr(ty))
+    if rc != 0:
+        raise RuntimeError(f"rmsnorm_jvp_f64 failed with code {rc}")
+    return y, ty

@@ -22,7 +22,7 @@ ERR_STATIC_SCRATCH = 13
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 EXPORTS = ("attn_jvp_fwd", "attn_jvp_fwd_stream", "attn_jvp_fwd_mu", "attn_jvp_splitkv_workspace_bytes",
-           "attn_jvp_fwd_splitkv", "attn_jvp_fwd_splitkv_static", "attn_jvp_selftest_bounded_wait", "attn_jvp_set_stream", "attn_jvp_device_status", "attn_jvp_strerror",
+           "attn_jvp_fwd_splitkv", "attn_jvp_fwd_splitkv_static", "attn_jvp_qknorm_fwd", "attn_jvp_selftest_bounded_wait", "attn_jvp_set_stream", "attn_jvp_device_status", "attn_jvp_strerror",
            "attn_jvp_version")
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libattn_jvp.so")
@@ -64,6 +64,8 @@ def load():
             lib.attn_jvp_fwd_splitkv.restype = ci
             lib.attn_jvp_fwd_splitkv_static.argtypes = [vp] * 10 + [ci] * 5 + [cf, cu, ci, vp]
             lib.attn_jvp_fwd_splitkv_static.restype = ci
+            lib.attn_jvp_qknorm_fwd.argtypes = [vp] * 5 + [ctypes.c_longlong, ci, cf, vp]
+            lib.attn_jvp_qknorm_fwd.restype = ci
             lib.attn_jvp_selftest_bounded_wait.argtypes = [vp]
             lib.attn_jvp_selftest_bounded_wait.restype = ci
             lib.attn_jvp_set_stream.argtypes = [vp]
@@ -145,6 +147,32 @@ def attn_jvp_fwd_splitkv_static(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, L
     return int(load().attn_jvp_fwd_splitkv_static(_ptr(q), _ptr(k), _ptr(v), _ptr(tq), _ptr(tk), _ptr(tv), _ptr(o),
                                                   _ptr(to), _ptr(lse), _ptr(mu), B, H, Lq, Lk, D, float(scale),
                                                   int(flags), int(splits), _ptr(cuda_stream)))
+
+
+def attn_jvp_qknorm_fwd(x, tx, w, y, ty, rows, D, eps, cuda_stream) -> int:
+    """Raw call of the RMS-norm JVP kernel: tensors or device addresses in, return code out."""
+    return int(load().attn_jvp_qknorm_fwd(_ptr(x), _ptr(tx), _ptr(w), _ptr(y), _ptr(ty), int(rows), int(D),
+                                          float(eps), _ptr(cuda_stream)))
+
+
+def qknorm_jvp(x, tx, w, eps=1e-6):
+    """y = w . x / rms(x) over the last dimension and its tangent ty for tangent tx (None: primal only).
+
+    x, tx: contiguous CUDA bf16 tensors [..., D]; w: CUDA fp32 [D].  Returns (y, ty)."""
+    if not (x.is_cuda and x.dtype == torch.bfloat16 and x.is_contiguous()):
+        raise ValueError("x must be a contiguous CUDA bf16 tensor")
+    if tx is not None and not (tx.is_cuda and tx.dtype == torch.bfloat16 and tx.is_contiguous() and tx.shape == x.shape):
+        raise ValueError("tx must match x")
+    D = x.shape[-1]
+    if not (w.is_cuda and w.dtype == torch.float32 and w.is_contiguous() and tuple(w.shape) == (D,)):
+        raise ValueError("w must be a contiguous CUDA fp32 tensor of shape [D]")
+    y = torch.empty_like(x)
+    ty = None if tx is None else torch.empty_like(x)
+    with torch.cuda.device(x.device):
+        rc = attn_jvp_qknorm_fwd(x, tx, w, y, ty, x.numel() // D, D, eps, torch.cuda.current_stream().cuda_stream)
+    if rc != 0:
+        raise AttnJvpError(rc, attn_jvp_strerror(rc))
+    return y, ty
 
 
 def _check(t, name, shape):

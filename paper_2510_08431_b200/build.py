@@ -8,7 +8,8 @@ import subprocess
 PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 SRC = os.path.join(PKG, "csrc", "attn_jvp.cu")
-DEPS = [SRC, os.path.join(PKG, "csrc", "attn_jvp_kernel.cuh"), os.path.join(ROOT, "include", "attn_jvp.h")]
+DEPS = [SRC, os.path.join(PKG, "csrc", "attn_jvp_kernel.cuh"), os.path.join(PKG, "csrc", "qknorm_jvp.cuh"),
+        os.path.join(ROOT, "include", "attn_jvp.h")]
 LIB = os.path.join(PKG, "libattn_jvp.so")
 
 

@@ -8,6 +8,7 @@
 #include <cstring>
 
 #include "attn_jvp_kernel.cuh"
+#include "qknorm_jvp.cuh"
 
 namespace {
 
@@ -324,6 +325,47 @@ int attn_jvp_fwd_splitkv_static(const void* q, const void* k, const void* v, con
     }
     return run(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, Lk, D, scale, flags, splits, g_static_scratch_dev[dev],
                (size_t)ATTN_JVP_STATIC_SCRATCH_BYTES, static_cast<cudaStream_t>(cuda_stream), /*may_allocate=*/false);
+}
+
+int attn_jvp_qknorm_fwd(const void* x, const void* tx, const float* w, void* y, void* ty, long long rows, int D,
+                        float eps, void* cuda_stream) {
+    if (rows < 1) return ATTN_JVP_ERR_SHAPE;
+    if (D != 64 && D != 128) return ATTN_JVP_ERR_UNSUPPORTED_D;
+    if (!x || !w || !y) return ATTN_JVP_ERR_NULL;
+    if ((tx == nullptr) != (ty == nullptr)) return ATTN_JVP_ERR_NULL;     // tangent in and out go together
+    if (!std::isfinite(eps) || eps < 0.0f) return ATTN_JVP_ERR_SCALE;
+    const void* ptrs[5] = {x, tx, w, y, ty};
+    for (const void* p : ptrs) if (p && ((uintptr_t)p & 15u)) return ATTN_JVP_ERR_ALIGN;
+    const size_t bytes = (size_t)rows * D * 2;
+    if (overlaps(y, bytes, x, bytes) || overlaps(y, bytes, tx, bytes) || overlaps(ty, bytes, x, bytes) ||
+        overlaps(ty, bytes, tx, bytes) || overlaps(y, bytes, ty, bytes) || overlaps(y, bytes, w, (size_t)D * 4) ||
+        overlaps(ty, bytes, w, (size_t)D * 4))
+        return ATTN_JVP_ERR_ALIAS;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail("cudaGetDevice", e);
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return cuda_fail("cudaDeviceGetAttribute(MultiProcessorCount)", e);
+    const int rows_per_block = 256 / (D / 8);
+    long long blocks = (rows + rows_per_block - 1) / rows_per_block;
+    const long long cap = (long long)sms * 16;                 // a multiple of the SM count; the kernel strides
+    if (blocks > cap) blocks = cap;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const uint4* xp = static_cast<const uint4*>(x);
+    const uint4* tp = static_cast<const uint4*>(tx);
+    uint4* yp = static_cast<uint4*>(y);
+    uint4* typ = static_cast<uint4*>(ty);
+    if (D == 128) {
+        if (tx) attn_jvp::qknorm_jvp_kernel<128, true><<<(unsigned)blocks, 256, 0, st>>>(xp, tp, w, yp, typ, rows, eps);
+        else attn_jvp::qknorm_jvp_kernel<128, false><<<(unsigned)blocks, 256, 0, st>>>(xp, tp, w, yp, typ, rows, eps);
+    } else {
+        if (tx) attn_jvp::qknorm_jvp_kernel<64, true><<<(unsigned)blocks, 256, 0, st>>>(xp, tp, w, yp, typ, rows, eps);
+        else attn_jvp::qknorm_jvp_kernel<64, false><<<(unsigned)blocks, 256, 0, st>>>(xp, tp, w, yp, typ, rows, eps);
+    }
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail("qknorm kernel launch", e);
+    return 0;
 }
 
 int attn_jvp_selftest_bounded_wait(void* cuda_stream) {

@@ -81,3 +81,22 @@ def test_splitkv_workspace_checks(aj):
     o1, to1, lse1 = aj.attention_jvp(g["q"], g["k"], g["v"], g["tq"], g["tk"], g["tv"])
     torch.cuda.synchronize()
     assert (o.float() - o1.float()).abs().max() <= 4e-3 and (to.float() - to1.float()).abs().max() <= 8e-3
+
+
+def test_layer_front_end_matches_direct_calls(aj):
+    """The withT protocol of the layer wrapper is argument routing only."""
+    B, H, Lq, Lk, D = 1, 2, 200, 300, 128
+    x = synth.make_inputs(B, H, Lq, Lk, D, 1.0, 0.5, seed=63)
+    g = U.to_gpu(x)
+    layer = aj.AttentionCoreJVP(scale=0.1, keep_mu=True)
+    o_plain = layer(g["q"], g["k"], g["v"])
+    o, to = layer((g["q"], g["tq"]), (g["k"], g["tk"]), (g["v"], g["tv"]), withT=True)
+    lse, mu = layer.last_lse, layer.last_mu
+    oc, toc = layer((g["q"], g["tq"]), g["k"], g["v"], withT=True)          # constant context
+    ro, rto, rlse, rmu = aj.attention_jvp(g["q"], g["k"], g["v"], g["tq"], g["tk"], g["tv"], scale=0.1, return_mu=True)
+    rco, rcto, _ = aj.attention_jvp(g["q"], g["k"], g["v"], g["tq"], None, None, scale=0.1)
+    torch.cuda.synchronize()
+    assert torch.equal(o, ro) and torch.equal(to, rto) and torch.equal(lse, rlse) and torch.equal(mu, rmu)
+    assert torch.equal(o_plain, ro) and torch.equal(oc, rco) and torch.equal(toc, rcto)
+    with pytest.raises(ValueError):
+        layer((g["q"], g["tq"]), (g["k"], g["tk"]), g["v"], withT=True)
