@@ -166,6 +166,59 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
+def run_qknorm(args, w, aj):
+    """Side benchmark of the RMS-norm JVP kernel on the q tensor of the workload: rows = B*Lq*H, memory bound."""
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (sm_100a); there is no CPU path")
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    g = torch.Generator(device="cpu").manual_seed(w.seed)
+    x = torch.randn((w.B, w.Lq, w.H, w.D), generator=g).to(torch.bfloat16).to(dev)
+    tx = (torch.randn((w.B, w.Lq, w.H, w.D), generator=g) * w.sigma_tangent).to(torch.bfloat16).to(dev)
+    wt = torch.ones(w.D, device=dev)
+    rows = w.B * w.Lq * w.H
+    nbytes = 4 * rows * w.D * 2
+    flush = torch.empty(512 * 1024 * 1024, dtype=torch.uint8, device=dev) if nbytes <= 2 * 126e6 else None
+    y = torch.empty_like(x); ty = torch.empty_like(x)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        rc = aj.attn_jvp_qknorm_fwd(x, tx, wt, y, ty, rows, w.D, 1e-6, stream.cuda_stream)
+        if rc != 0:
+            raise RuntimeError(aj.attn_jvp_strerror(rc))
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for a, b in evs:
+        if flush is not None:
+            flush.zero_()
+        a.record(stream); step(); b.record(stream)
+    torch.cuda.synchronize()
+    ms = [a.elapsed_time(b) for a, b in evs]
+    mean_ms = sum(ms) / len(ms)
+    hbm = 6549.1
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    src = "fallback"
+    if os.path.exists(path):
+        with open(path) as f:
+            hbm = float(json.load(f)["hbm_gbs"]); src = "measured"
+    else:
+        hbm = 6650.0
+    achieved = nbytes / (mean_ms * 1e-3) / 1e9
+    line = {"metric": "qknorm-JVP GB/s (4 tensors x rows x D x 2 B)", "value": achieved, "unit": "GB/s", "n_gpus": 1,
+            "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": mean_ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"qknorm on the q tensor of {w.name}", "rows": rows, "D": w.D,
+                       "l2": "tensors larger than L2" if flush is None else "L2 flushed between timed iterations"},
+            "gpu_launches": args.steps,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": hbm, "unit": "GB/s", "frac": achieved / hbm,
+                         "traffic": None, "peak_source": f"{src} copy bandwidth", "kernel": "qknorm_jvp_kernel",
+                         "algorithmic_bytes": nbytes}}
+    print(json.dumps(line), flush=True)
+
+
 def workload_config(w, extra=None):
     cfg = {"workload": w.name, "B": w.B, "H": w.H, "Lq": w.Lq, "Lk": w.Lk, "D": w.D, "scale": w.scale,
            "kv_tangent_free": w.kv_tangent_free, "layout": "BLHD bf16", "seed": w.seed,
@@ -186,6 +239,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--splits", type=int, default=1, help="key chunks (split-KV entry point) for few-query workloads")
+    ap.add_argument("--op", default="attention", choices=["attention", "qknorm"],
+                    help="attention = the hot path (default); qknorm = the RMS-norm JVP that feeds it (memory bound)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = synth.WORKLOADS[args.workload]
@@ -196,6 +251,9 @@ def main():
 
     import paper_2510_08431_b200 as aj
     aj.load()   # raises if the CUDA library is missing: there is no fallback
+    if args.op == "qknorm":
+        run_qknorm(args, w, aj)
+        return
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
