@@ -16,6 +16,7 @@ using attn_jvp::KernelArgs;
 
 constexpr int kVersion = 100;   // 0.1.0
 constexpr int kMaxDevices = 64;
+constexpr int kPersistentMaxTiles = 128;   // key tiles per work item up to which CTAs are persistent
 
 thread_local cudaStream_t tl_stream = nullptr;
 thread_local char tl_cuda_msg[256] = "";
@@ -23,6 +24,7 @@ thread_local char tl_strerror_buf[384];
 
 int* g_host_status[kMaxDevices] = {};       // mapped pinned host words, one per device
 int* g_host_status_dev[kMaxDevices] = {};   // their device-side addresses
+int g_sm_count[kMaxDevices] = {};
 int g_dyn_smem[kMaxDevices][2][3][2] = {};  // dynamic shared memory per kernel instantiation, 0 = not set up
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -225,7 +227,25 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
         ka.part_mu = reinterpret_cast<float*>(w + 2 * lay.vec_bytes + lay.stat_bytes);
     }
 
-    const dim3 grid((Lq + attn_jvp::kBlockM - 1) / attn_jvp::kBlockM, H, B * eff_splits);
+    // persistent CTAs: one per SM (fewer if there is less work), sharing the work items round-robin
+    const long long n_q_tiles = (Lq + attn_jvp::kBlockM - 1) / attn_jvp::kBlockM;
+    const long long n_items = n_q_tiles * H * B * eff_splits;
+    if (n_items > 0x7fffffffLL) return ATTN_JVP_ERR_SHAPE;
+    ka.n_q_tiles = (int)n_q_tiles;
+    ka.n_items = (int)n_items;
+    if (g_sm_count[dev] == 0) {
+        int sms = 0;
+        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return cuda_fail("cudaDeviceGetAttribute(MultiProcessorCount)", e);
+        g_sm_count[dev] = sms;
+    }
+    // Short items (few key tiles): one persistent CTA per SM, so that the epilogue of an item overlaps the
+    // start of the next.  Long items: one CTA per item, which lets the hardware balance the load (a static
+    // round-robin costs up to one item of imbalance at the end, which is more than the overlap saves there).
+    const int tiles_per_item = split ? tiles_per_split : ka.n_kv_tiles;
+    const bool persistent = tiles_per_item <= kPersistentMaxTiles;
+    const long long n_ctas = (persistent && n_items > g_sm_count[dev]) ? g_sm_count[dev] : n_items;
+    const dim3 grid((unsigned)n_ctas, 1, 1);
     int rc;
 #define ATTN_JVP_DISPATCH(DD, SS)                                                                                  \
     switch (mode) {                                                                                               \

@@ -1,17 +1,16 @@
 // Attention-JVP forward kernel for sm_100a (Algorithm 2: FlashAttention-2 forward with JVP).
 //
 // One CTA owns a 128-row query tile of one (batch, head) and streams the keys in
-// tiles of 64.  Roles (warp-specialised, 64 + 128*kGroups threads):
+// tiles of 64; CTAs are persistent (one per SM) and walk the query tiles round-robin, so that the epilogue of
+// one tile overlaps the loads and the first score MMAs of the next.  Roles (warp-specialised, 192 threads):
 //   warp 0     MMA issuer: the whole warp runs the loop in lock step, one elected lane issues
 //              tcgen05.mma with accumulators in tensor memory.
-//   warp 1     TMA producer: Q,tQ once, then K|tK and V|tV tiles into a shared-memory ring.
-//   warps 2..  softmax: kGroups groups of four warps; thread (w, lane) owns query row
-//              32*(w%4) + lane (its tensor-memory lane) and 64/kGroups columns of every score tile.
-//              Reads S and tS from tensor memory, keeps m, l, r (Algorithm 2 lines 10-12, 16) in
-//              registers, writes P~ and H~ = P~ . tS back to tensor memory as bf16 MMA operands,
-//              rescales the accumulators when the running max moves, and runs the epilogue
-//              (lines 19-23).  With kGroups = 2 the two owners of a row exchange the row max through
-//              shared memory and their partial sums through dead tensor-memory columns.
+//   warp 1     TMA producer: Q,tQ per query tile, K|tK and V|tV tiles into a shared-memory ring.
+//   warps 2-5  softmax: thread (w, lane) owns query row 32*(w%4) + lane (its tensor-memory lane) and
+//              all 64 columns of every score tile.  Reads S and tS from tensor memory, keeps m, l, r
+//              (Algorithm 2 lines 10-12, 16) in registers, writes P~ and H~ = P~ . tS back to tensor
+//              memory as bf16 MMA operands, rescales the accumulators when the running max moves, and
+//              runs the epilogue (lines 19-23).
 //
 // Tensor-memory map (512 columns x 128 lanes, fp32):
 //   [0, D)        O  accumulator (line 13)
@@ -36,16 +35,11 @@ namespace attn_jvp {
 
 constexpr int kBlockM = 128;        // query rows per CTA (B_r)
 constexpr int kBlockN = 64;         // keys per tile (B_c)
-#ifndef ATTN_JVP_SOFTMAX_GROUPS
-#define ATTN_JVP_SOFTMAX_GROUPS 1     // measured: one group of four warps is as fast as two and needs no exchange
-#endif
-constexpr int kGroups = ATTN_JVP_SOFTMAX_GROUPS;   // groups of four softmax warps; each owns 64/kGroups columns of a score tile
-constexpr int kSoftmaxThreads = 128 * kGroups;
+constexpr int kSoftmaxThreads = 128;   // four softmax warps: one thread per query row
 constexpr int kMmaWarp = 0;            // the two single-thread roles come first (oldest warps of the CTA)
 constexpr int kProducerWarp = 1;
 constexpr int kFirstSoftmaxWarp = 2;
 constexpr int kThreads = kSoftmaxThreads + 64;
-constexpr int kHalfN = kBlockN / kGroups;      // score columns per softmax thread
 constexpr int kTmemCols = 512;
 constexpr int kScoreCol0 = 256;     // first column of score buffer 0
 constexpr int kScoreBufStride = 128;
@@ -93,6 +87,8 @@ struct KernelArgs {
     float* part_lse;    // [splits][B][H][Lq]
     float* part_mu;     // [splits][B][H][Lq]
     int B;
+    int n_q_tiles;      // 128-row query tiles per (batch, head)
+    int n_items;        // work items = n_q_tiles * H * B * splits; the grid's CTAs share them round-robin
 };
 
 template <int D>
@@ -353,32 +349,41 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     constexpr bool kHasTKV = (MODE == kModeJvp);             // tK, tV are read
 
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_q_full;
+    __shared__ __align__(8) uint64_t bar_q_full;     // Q, tQ of the current work item are in shared memory
+    __shared__ __align__(8) uint64_t bar_q_free;     // every score MMA of the item has completed: Q, tQ may be replaced
     __shared__ __align__(8) uint64_t bar_slot_full[kSlots];
     __shared__ __align__(8) uint64_t bar_slot_empty[kSlots];
     __shared__ __align__(8) uint64_t bar_s_full[2];
     __shared__ __align__(8) uint64_t bar_p_full[2];
     __shared__ __align__(8) uint64_t bar_pv_done;
+    __shared__ __align__(8) uint64_t bar_acc_free;   // the epilogue has read O and T: the next item may overwrite them
     __shared__ __align__(8) uint64_t bar_drain;
-    // Exchanges between the two warps that own the same 32 rows (quarter q = warp % 4): [0][q], [1][q] row
-    // maxima of even / odd key tiles, [2][q] partial sums.  One elected lane per warp arrives.
-    __shared__ __align__(8) uint64_t bar_xchg[3][4];
     __shared__ uint32_t tmem_base_smem;
     __shared__ int cta_abort;
-    __shared__ float xchg_max[2][2][kBlockM];     // [tile parity][column half][row]: per-half row maxima
 
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0);   // warp-uniform by construction
     const int lane = threadIdx.x & 31;
-    const int q_tile = blockIdx.x;
-    const int h = blockIdx.y;
-    const int b = kSplit ? blockIdx.z / args.splits : blockIdx.z;
-    const int split = kSplit ? blockIdx.z % args.splits : 0;
-    const int tile0 = kSplit ? split * args.tiles_per_split : 0;       // first key tile of this CTA
-    const int q0 = q_tile * kBlockM;
-    const int n_kv = kSplit ? min(args.tiles_per_split, args.n_kv_tiles - tile0) : args.n_kv_tiles;
 #ifdef ATTN_JVP_TRACE
-    const bool trace_on = blockIdx.x == gridDim.x / 2 && blockIdx.y == gridDim.y / 2 && blockIdx.z == 0;
+    const bool trace_on = blockIdx.x == gridDim.x / 2;
 #endif
+
+    // A CTA is persistent: it walks the work items blockIdx.x, blockIdx.x + gridDim.x, ... in the same order in
+    // every role.  An item is one 128-row query tile of one (batch, head[, key chunk]); query tiles vary fastest
+    // so that the CTAs running at one time share one head's K/V in L2.
+    struct Item { int q0, h, b, split, tile0, n_kv; };
+    auto decode = [&](int item) -> Item {
+        Item w;
+        w.q0 = (item % args.n_q_tiles) * kBlockM;
+        const int rest = item / args.n_q_tiles;
+        w.h = rest % args.H;
+        const int z = rest / args.H;
+        w.b = kSplit ? z / args.splits : z;
+        w.split = kSplit ? z % args.splits : 0;
+        w.tile0 = kSplit ? w.split * args.tiles_per_split : 0;       // first key tile of this item
+        w.n_kv = kSplit ? min(args.tiles_per_split, args.n_kv_tiles - w.tile0) : args.n_kv_tiles;
+        return w;
+    };
+    const int n_items = args.n_items;
 
     // An earlier CTA of this (or a previous) launch gave up: do not start.  One thread reads
     // the flag so that the whole CTA takes the same decision.
@@ -409,6 +414,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&bar_q_full), 1);
+        mbar_init(smem_u32(&bar_q_free), 1);
         for (int i = 0; i < kSlots; ++i) {
             mbar_init(smem_u32(&bar_slot_full[i]), 1);
             mbar_init(smem_u32(&bar_slot_empty[i]), 1);
@@ -418,9 +424,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             mbar_init(smem_u32(&bar_p_full[i]), kSoftmaxThreads / 32);    // one arrival per softmax warp
         }
         mbar_init(smem_u32(&bar_pv_done), 1);
+        mbar_init(smem_u32(&bar_acc_free), kSoftmaxThreads / 32);
         mbar_init(smem_u32(&bar_drain), 1);
-        for (int i = 0; i < 3; ++i)
-            for (int q = 0; q < 4; ++q) mbar_init(smem_u32(&bar_xchg[i][q]), 2);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kMmaWarp) {
@@ -442,23 +447,23 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const uint32_t tmem_o = tmem;
     const uint32_t tmem_t = tmem + D;
 
+    // Phases.  Key tiles are numbered g = 0, 1, 2, ... over ALL items of this CTA; tile g uses score buffer g & 1,
+    // phase (g >> 1) & 1 of bar_s_full / bar_p_full and phase g & 1 of bar_pv_done.  Item number `it` (0, 1, ...)
+    // uses phase it & 1 of bar_q_full / bar_q_free / bar_acc_free.  The shared-memory ring runs on without a break.
+
     if (warp == kProducerWarp) {
         // =====================================================================================
-        // TMA producer.  Ring order = consumption order: K0, K1, V0, K2, V1, ..., K(n-1), V(n-2), V(n-1).
+        // TMA producer.  Per item: Q, tQ (once the previous item's score MMAs are done), then the ring in
+        // consumption order K0, K1, V0, K2, V1, ..., K(n-1), V(n-2), V(n-1).
         // =====================================================================================
         if (lane == 0) {
             constexpr uint32_t kQTx = (kHasTQ ? 2u : 1u) * Plan::kQBytes;
             constexpr uint32_t kKTx = (kHasTKV ? 2u : 1u) * kHalves * Plan::kKvHalfBytes;
             constexpr uint32_t kVTx = kKTx;
             const uint32_t qbar = smem_u32(&bar_q_full);
-            mbar_arrive_expect_tx(qbar, kQTx);
-#pragma unroll
-            for (int hf = 0; hf < kHalves; ++hf) {
-                tma_load_4d(smem_q + hf * Plan::kQHalfBytes, &tm_q, qbar, hf * 64, h, q0, b);
-                if (kHasTQ) tma_load_4d(smem_tq + hf * Plan::kQHalfBytes, &tm_tq, qbar, hf * 64, h, q0, b);
-            }
             int t = 0;          // ring position
             bool ok = true;
+            Item w{};
             auto acquire = [&](uint32_t& slot_addr, uint32_t& bar) -> bool {
                 const int slot = t % kSlots;
                 if (t >= kSlots) {
@@ -477,9 +482,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 // per 64-column half: [K_half (8 KB)][tK_half (8 KB)] so that [K ; tK] is one N = 128 operand
 #pragma unroll
                 for (int hf = 0; hf < kHalves; ++hf) {
-                    tma_load_4d(dst + hf * 2 * Plan::kKvHalfBytes, &tm_k, bar, hf * 64, h, (tile0 + j) * kBlockN, b);
+                    tma_load_4d(dst + hf * 2 * Plan::kKvHalfBytes, &tm_k, bar, hf * 64, w.h, (w.tile0 + j) * kBlockN, w.b);
                     if (kHasTKV)
-                        tma_load_4d(dst + hf * 2 * Plan::kKvHalfBytes + Plan::kKvHalfBytes, &tm_tk, bar, hf * 64, h, (tile0 + j) * kBlockN, b);
+                        tma_load_4d(dst + hf * 2 * Plan::kKvHalfBytes + Plan::kKvHalfBytes, &tm_tk, bar, hf * 64, w.h, (w.tile0 + j) * kBlockN, w.b);
                 }
                 return true;
             };
@@ -490,19 +495,31 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 // [V_half0][V_half1][tV_half0][tV_half1]: consecutive 64-wide N atoms of [V | tV]
 #pragma unroll
                 for (int hf = 0; hf < kHalves; ++hf) {
-                    tma_load_4d(dst + hf * Plan::kKvHalfBytes, &tm_v, bar, hf * 64, h, (tile0 + j) * kBlockN, b);
+                    tma_load_4d(dst + hf * Plan::kKvHalfBytes, &tm_v, bar, hf * 64, w.h, (w.tile0 + j) * kBlockN, w.b);
                     if (kHasTKV)
-                        tma_load_4d(dst + (kHalves + hf) * Plan::kKvHalfBytes, &tm_tv, bar, hf * 64, h, (tile0 + j) * kBlockN, b);
+                        tma_load_4d(dst + (kHalves + hf) * Plan::kKvHalfBytes, &tm_tv, bar, hf * 64, w.h, (w.tile0 + j) * kBlockN, w.b);
                 }
                 return true;
             };
-            ok = load_k(0);
-            for (int j = 0; ok && j < n_kv; ++j) {
-                if (j + 1 < n_kv) ok = load_k(j + 1);
-                if (ok) ok = load_v(j);
+            int it = 0;
+            for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
+                w = decode(item);
+                if (it > 0) ok = mbar_wait(smem_u32(&bar_q_free), (it - 1) & 1, abort_state);
+                if (!ok) break;
+                mbar_arrive_expect_tx(qbar, kQTx);
+#pragma unroll
+                for (int hf = 0; hf < kHalves; ++hf) {
+                    tma_load_4d(smem_q + hf * Plan::kQHalfBytes, &tm_q, qbar, hf * 64, w.h, w.q0, w.b);
+                    if (kHasTQ) tma_load_4d(smem_tq + hf * Plan::kQHalfBytes, &tm_tq, qbar, hf * 64, w.h, w.q0, w.b);
+                }
+                ok = load_k(0);
+                for (int j = 0; ok && j < w.n_kv; ++j) {
+                    if (j + 1 < w.n_kv) ok = load_k(j + 1);
+                    if (ok) ok = load_v(j);
+                }
             }
             if (!ok) {
-                // Abandoning the tile: let the copies already in flight land before the CTA exits.
+                // Abandoning the work: let the copies already in flight land before the CTA exits.
                 const int issued = t;
                 for (int u = (issued > kSlots ? issued - kSlots : 0); u < issued; ++u) {
                     const uint32_t bar = smem_u32(&bar_slot_full[u % kSlots]);
@@ -525,17 +542,16 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             constexpr uint32_t kIdescHV = make_idesc(D, true);                                 // H~ x V
             constexpr uint32_t kVLbo = Plan::kKvHalfBytes;   // bytes between 64-wide N atoms of a V slot
             const bool leader = elect_one();
-            bool ok = mbar_wait_warp(smem_u32(&bar_q_full), 0, abort_state);
+            bool ok = true;
             const uint32_t q_lo = make_desc_lo(smem_q, 16);
             const uint32_t tq_lo = make_desc_lo(smem_tq, 16);
 
             // The hardware queue in front of the tensor pipe is short (about eight instructions), and this
-            // warp competes for issue slots with two busy softmax warps, so whatever runs between two
-            // groups of MMAs is kept to a minimum: per key tile there is ONE blocking wait (P~/H~ of tile j)
-            // followed by one burst that issues the value MMAs of tile j and the score MMAs of tile j+2.
-            // The shared-memory slots those need were filled long before in steady state; they are tested
-            // first and waited for only if a test fails.  Ring position -> (slot, parity) is tracked
-            // incrementally.
+            // warp competes for issue slots with the softmax warps, so whatever runs between two
+            // groups of MMAs is kept to a minimum: per key tile there is ONE burst that issues the value MMAs
+            // of tile j and the score MMAs of tile j+2, and the barriers the NEXT burst depends on are tested in
+            // the middle of it, while the queue is still full.  Only if a test fails does the warp block.
+            // Ring position -> (slot, parity) is tracked incrementally.
             struct RingPos { int slot; uint32_t parity; };
             auto advance = [&](RingPos& r) { if (++r.slot == kSlots) { r.slot = 0; r.parity ^= 1u; } };
             auto wait_full = [&](const RingPos& r) -> bool {
@@ -545,9 +561,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             };
 
             // Operand descriptors.  Q and tQ never move: their eight per-k-step descriptors are built once.
-            // Those of a ring slot are built by prepare_*() BEFORE the burst that uses them (while the warp
-            // would be waiting for queue space anyway), so that inside a burst every tcgen05.mma is a single
-            // instruction with its operands ready.
+            // Those of a ring slot are built by prepare_*() BEFORE the burst that uses them, so that inside a
+            // burst every tcgen05.mma is a single instruction with its operands ready.
             uint64_t qd[D / 16], tqd[D / 16];
 #pragma unroll
             for (int k = 0; k < D / 16; ++k) {
@@ -569,17 +584,17 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 for (int k = 0; k < kBlockN / 16; ++k) vd[k] = make_desc(v_lo + k * (2048 >> 4));
             };
 
-            // score MMAs of tile j (issued by the elected lane), in two parts so that the look-ahead for the
-            // next tile can run between them
-            auto issue_scores_a = [&](int j) {
-                const uint32_t tm_s = tmem + kScoreCol0 + (j & 1) * kScoreBufStride;
-                TRACE(21, j);         // MMA: about to issue score MMAs
+            // score MMAs of global tile g (issued by the elected lane), in two parts so that the look-ahead for
+            // the next tile can run between them; `last_of_item`: these are the item's last score MMAs
+            auto issue_scores_a = [&](int g) {
+                const uint32_t tm_s = tmem + kScoreCol0 + (g & 1) * kScoreBufStride;
+                TRACE(21, g);         // MMA: about to issue score MMAs
                 mma_ss<false>(tm_s, qd[0], kd[0], kIdescS1);
 #pragma unroll
                 for (int k = 1; k < D / 16; ++k) mma_ss<true>(tm_s, qd[k], kd[k], kIdescS1);
             };
-            auto issue_scores_b = [&](int j, int slot) {
-                const uint32_t tm_ts = tmem + kScoreCol0 + (j & 1) * kScoreBufStride + kBlockN;
+            auto issue_scores_b = [&](int g, int slot, bool last_of_item) {
+                const uint32_t tm_ts = tmem + kScoreCol0 + (g & 1) * kScoreBufStride + kBlockN;
                 if (kHasTQ) {
                     if (kHasTKV) mma_ss<true>(tm_ts, tqd[0], kd[0], kIdescS2);
                     else mma_ss<false>(tm_ts, tqd[0], kd[0], kIdescS2);
@@ -587,14 +602,15 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     for (int k = 1; k < D / 16; ++k) mma_ss<true>(tm_ts, tqd[k], kd[k], kIdescS2);
                 }
                 tc_commit(smem_u32(&bar_slot_empty[slot]));
-                tc_commit(smem_u32(&bar_s_full[j & 1]));
-                TRACE(2, j);          // MMA: score MMAs of tile j issued
+                tc_commit(smem_u32(&bar_s_full[g & 1]));
+                if (last_of_item) tc_commit(smem_u32(&bar_q_free));
+                TRACE(2, g);          // MMA: score MMAs of tile g issued
             };
-            // value MMAs of tile j out of ring slot `slot`
-            auto issue_values = [&](int j, int slot) {
-                const uint32_t tm_p = tmem + kScoreCol0 + (j & 1) * kScoreBufStride;
+            // value MMAs of tile j of the item (global tile g) out of ring slot `slot`
+            auto issue_values = [&](int j, int g, int slot) {
+                const uint32_t tm_p = tmem + kScoreCol0 + (g & 1) * kScoreBufStride;
                 const uint32_t tm_h = tm_p + kBlockN;
-                TRACE(3, j);          // MMA: about to issue value MMAs
+                TRACE(3, g);          // MMA: about to issue value MMAs
 #pragma unroll
                 for (int k = 0; k < kBlockN / 16; ++k) {
                     mma_ts(tmem_o, tm_p + k * 8, vd[k], kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
@@ -607,87 +623,94 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
                 tc_commit(smem_u32(&bar_slot_empty[slot]));
                 tc_commit(smem_u32(&bar_pv_done));
-                TRACE(4, j);          // MMA: value MMAs of tile j issued
+                TRACE(4, g);          // MMA: value MMAs of tile g issued
             };
-            // what tile j's burst needs: V(j) and K(j+2) in shared memory, P~/H~ of tile j in tensor memory
-            auto test_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, int j) -> bool {
+            // what the burst of global tile g needs: V and K(+2) in shared memory, P~/H~ in tensor memory
+            auto test_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, int g) -> bool {
                 bool r = mbar_test_wait(smem_u32(&bar_slot_full[pv.slot]), pv.parity);
                 if (has_k) r = r && mbar_test_wait(smem_u32(&bar_slot_full[pk.slot]), pk.parity);
-                r = r && mbar_test_wait(smem_u32(&bar_p_full[j & 1]), (j >> 1) & 1);
+                r = r && mbar_test_wait(smem_u32(&bar_p_full[g & 1]), (g >> 1) & 1);
                 return __all_sync(0xffffffffu, r);
             };
-            auto wait_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, int j) -> bool {
-                if (leader) TRACE(22, j);   // MMA: has to block for tile j
+            auto wait_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, int g) -> bool {
+                if (leader) TRACE(22, g);   // MMA: has to block for tile g
                 bool r = wait_full(pv);
                 if (r && has_k) r = wait_full(pk);
-                if (r) r = mbar_wait_warp(smem_u32(&bar_p_full[j & 1]), (j >> 1) & 1, abort_state);
+                if (r) r = mbar_wait_warp(smem_u32(&bar_p_full[g & 1]), (g >> 1) & 1, abort_state);
                 return r;
             };
 
-            // Ring order (as the producer fills it): K0, K1, V0, K2, V1, K3, ...
+            // Ring order (as the producer fills it), per item: K0, K1, V0, K2, V1, K3, ...
             RingPos pos{0, 0u};
-            if (ok) ok = wait_full(pos);
-            if (ok) {
+            int g0 = 0;          // global number of the item's first key tile
+            int it = 0;
+            for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
+                const Item w = decode(item);
+                const int n_kv = w.n_kv;
+                ok = mbar_wait_warp(smem_u32(&bar_q_full), it & 1, abort_state);
+                if (ok) ok = wait_full(pos);
+                if (!ok) break;
                 tc_fence_after();
                 prepare_k(pos.slot);
-                if (leader) { issue_scores_a(0); issue_scores_b(0, pos.slot); }
+                if (leader) { issue_scores_a(g0); issue_scores_b(g0, pos.slot, n_kv == 1); }
                 __syncwarp();
                 advance(pos);
-            }
-            if (ok && n_kv > 1) {
-                ok = wait_full(pos);
-                if (ok) {
+                if (n_kv > 1) {
+                    ok = wait_full(pos);
+                    if (!ok) break;
                     prepare_k(pos.slot);
-                    if (leader) { issue_scores_a(1); issue_scores_b(1, pos.slot); }
+                    if (leader) { issue_scores_a(g0 + 1); issue_scores_b(g0 + 1, pos.slot, n_kv == 2); }
                     __syncwarp();
                     advance(pos);
                 }
-            }
-            // pos = V(0).  Per tile j: burst = value MMAs of tile j, score MMAs of tile j+2; the barriers of tile
-            // j+1 are tested in the middle of the burst, while the queue is still full.
-            RingPos pos_v = pos, pos_k = pos;
-            bool has_k = n_kv > 2;
-            if (ok) {
+                // pos = V(0).  Per tile j: burst = value MMAs of tile j, score MMAs of tile j+2; the barriers of
+                // tile j+1 are tested in the middle of the burst, while the queue is still full.
+                RingPos pos_v = pos, pos_k = pos;
+                bool has_k = n_kv > 2;
                 advance(pos);
                 pos_k = pos;
                 if (has_k) advance(pos);
-                ok = wait_tile(pos_v, pos_k, has_k, 0);
+                ok = wait_tile(pos_v, pos_k, has_k, g0);
+                // the first value MMA of an item overwrites O and T: the previous item's epilogue must have read them
+                if (ok && it > 0) ok = mbar_wait_warp(smem_u32(&bar_acc_free), (it - 1) & 1, abort_state);
+                if (!ok) break;
                 prepare_v(pos_v.slot);
                 if (has_k) prepare_k(pos_k.slot);
-            }
-            for (int j = 0; ok && j < n_kv; ++j) {
-                // ring positions of the next tile
-                const RingPos nxt_v = pos;
-                RingPos nxt_k = pos;
-                const bool nxt_exists = j + 1 < n_kv;
-                const bool nxt_has_k = j + 3 < n_kv;
-                if (nxt_exists) {
-                    advance(pos);
-                    nxt_k = pos;
-                    if (nxt_has_k) advance(pos);
+                for (int j = 0; ok && j < n_kv; ++j) {
+                    // ring positions of the next tile
+                    const RingPos nxt_v = pos;
+                    RingPos nxt_k = pos;
+                    const bool nxt_exists = j + 1 < n_kv;
+                    const bool nxt_has_k = j + 3 < n_kv;
+                    if (nxt_exists) {
+                        advance(pos);
+                        nxt_k = pos;
+                        if (nxt_has_k) advance(pos);
+                    }
+                    tc_fence_after();
+                    if (leader) {
+                        issue_values(j, g0 + j, pos_v.slot);
+                        if (has_k) issue_scores_a(g0 + j + 2);
+                    }
+                    __syncwarp();
+                    bool nxt_ready = true;
+                    if (nxt_exists) nxt_ready = test_tile(nxt_v, nxt_k, nxt_has_k, g0 + j + 1);
+                    if (leader && has_k) issue_scores_b(g0 + j + 2, pos_k.slot, j + 3 == n_kv);
+                    __syncwarp();
+                    // descriptors of the next burst (this warp is held back by the full queue here anyway)
+                    if (nxt_exists) {
+                        prepare_v(nxt_v.slot);
+                        if (nxt_has_k) prepare_k(nxt_k.slot);
+                    }
+                    if (nxt_exists && !nxt_ready) ok = wait_tile(nxt_v, nxt_k, nxt_has_k, g0 + j + 1);
+                    pos_v = nxt_v;
+                    pos_k = nxt_k;
+                    has_k = nxt_has_k;
                 }
-                tc_fence_after();
-                if (leader) {
-                    issue_values(j, pos_v.slot);
-                    if (has_k) issue_scores_a(j + 2);
-                }
-                __syncwarp();
-                bool nxt_ready = true;
-                if (nxt_exists) nxt_ready = test_tile(nxt_v, nxt_k, nxt_has_k, j + 1);
-                if (leader && has_k) issue_scores_b(j + 2, pos_k.slot);
-                __syncwarp();
-                // descriptors of the next burst (this warp is held back by the full queue here anyway)
-                if (nxt_exists) {
-                    prepare_v(nxt_v.slot);
-                    if (nxt_has_k) prepare_k(nxt_k.slot);
-                }
-                if (nxt_exists && !nxt_ready) ok = wait_tile(nxt_v, nxt_k, nxt_has_k, j + 1);
-                pos_v = nxt_v;
-                pos_k = nxt_k;
-                has_k = nxt_has_k;
+                g0 += n_kv;
             }
             if (!ok && leader) {
-                // Abandoning the tile: wait (bounded) until the tensor core has drained what was issued.
+                // Abandoning the work: wait (bounded) until the tensor core has drained what was issued.
                 tc_commit(smem_u32(&bar_drain));
                 const unsigned long long t0 = globaltimer_ns();
                 while (!mbar_try_wait(smem_u32(&bar_drain), 0) && globaltimer_ns() - t0 < 100000000ull) {}
@@ -697,230 +720,190 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     } else {
         // =====================================================================================
         // Softmax warps.  Thread (warp w, lane) owns query row 32*(w%4) + lane (= its tensor-memory
-        // lane) and columns [32*half, 32*half + 32) of every score tile, half = (w - 2) / 4.
+        // lane) and all 64 columns of every score tile.
         // =====================================================================================
-        const int half = (warp - kFirstSoftmaxWarp) >> 2;
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;                          // 0..127: a warp may only touch lanes 32*(warp%4)..+31
-        const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
         const float c1 = args.scale_log2;
         const float sc = args.scale;
         const bool neg_scale = c1 < 0.0f;
-        float m_ref = -INFINITY;   // running reference max, log2 domain (m of Algorithm 2, lazily updated)
-        float l_run = 0.0f;        // this half's share of l
-        float r_run = 0.0f;        // this half's share of r (of the centred tS, see below)
-        float ts_shift = 0.0f;     // per-row constant subtracted from tS
         bool ok = true;
+        int g0 = 0;          // global number of the item's first key tile
+        int it = 0;
 
-        for (int j = 0; j < n_kv; ++j) {
-            const int bsel = j & 1;
-            if (!mbar_wait_warp(smem_u32(&bar_s_full[bsel]), (j >> 1) & 1, abort_state)) { ok = false; break; }
-            tc_fence_after();
-#if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
-            const bool trace_me = trace_on && lane == 0;
-            if (trace_me && j < kTraceSteps) g_trace[5 + (warp - kFirstSoftmaxWarp)][j] = clock64();     // softmax warp: scores seen ready
-#endif
-            const uint32_t tm_s = tmem + lane_base + kScoreCol0 + bsel * kScoreBufStride;
-            const uint32_t tm_ts = tm_s + kBlockN;
+        for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
+            const Item w = decode(item);
+            const int n_kv = w.n_kv;
+            float m_ref = -INFINITY;   // running reference max, log2 domain (m of Algorithm 2, lazily updated)
+            float l_run = 0.0f;        // l
+            float r_run = 0.0f;        // r (of the centred tS, see below)
+            float ts_shift = 0.0f;     // per-row constant subtracted from tS
 
-            uint32_t sv[kHalfN];
-            uint32_t tv[kHalfN];
-#pragma unroll
-            for (int c0 = 0; c0 < kHalfN; c0 += 32) {
-                TMEM_LD32(tm_s + half * kHalfN + c0, sv, c0);
-                if (kHasTQ) TMEM_LD32(tm_ts + half * kHalfN + c0, tv, c0);
-            }
-            tc_wait_ld();
-
-            // keys past Lk (zero-filled by TMA) must not enter the softmax
-            const int valid = args.Lk - (tile0 + j) * kBlockN - half * kHalfN;    // valid columns of this half
-            if (valid < kHalfN) {
-                const uint32_t masked = neg_scale ? 0x7F800000u : 0xFF800000u;   // -inf after scaling
-#pragma unroll
-                for (int c = 0; c < kHalfN; ++c) if (c >= valid) sv[c] = masked;
-            }
-
-            // rowmax(S_ij) of this half (four independent chains), in the log2 domain
-            float mx4[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) mx4[u] = __uint_as_float(sv[u]);
-            if (!neg_scale) {
-#pragma unroll
-                for (int c = 4; c < kHalfN; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(sv[c]));
-            } else {
-#pragma unroll
-                for (int c = 4; c < kHalfN; ++c) mx4[c & 3] = fminf(mx4[c & 3], __uint_as_float(sv[c]));
-            }
-            float mx = neg_scale ? fminf(fminf(mx4[0], mx4[1]), fminf(mx4[2], mx4[3]))
-                                 : fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-            mx *= c1;    // -inf when the whole half is masked (c1 == 0 gives NaN, which fmaxf below drops)
-            if (kGroups == 2) {
-                // exchange with the thread that owns the other half of this row
-                xchg_max[bsel][half][row] = mx;
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bar_xchg[bsel][quarter]));
-                if (!mbar_wait_warp(smem_u32(&bar_xchg[bsel][quarter]), (j >> 1) & 1, abort_state)) { ok = false; break; }
-                mx = fmaxf(mx, xchg_max[bsel][half ^ 1][row]);
-            }
-
-            // m_new = max(m, rowmax), applied lazily: the result does not depend on which
-            // reference is used as long as exp() stays in range.  Both owners of a row take
-            // the same decision from the same numbers.
-            float alpha = 1.0f;
-            const bool need = mx > m_ref + kRescaleThreshold;
-            if (need) {
-                alpha = ex2f(m_ref - mx);    // e^{m - m_new}; 0 on the first tile (m = -inf)
-                m_ref = mx;
-            }
-            if (j > 0 && __any_sync(0xffffffffu, need)) {
-                // the accumulators must be complete up to tile j-1 before they are rescaled
-                if (!mbar_wait_warp(smem_u32(&bar_pv_done), (j - 1) & 1, abort_state)) { ok = false; break; }
+            for (int j = 0; j < n_kv; ++j) {
+                const int g = g0 + j;
+                const int bsel = g & 1;
+                if (!mbar_wait_warp(smem_u32(&bar_s_full[bsel]), (g >> 1) & 1, abort_state)) { ok = false; break; }
                 tc_fence_after();
-                constexpr int kAccCols = kHasTQ ? 2 * D : D;     // each half rescales its share of the columns
-#pragma unroll 1
-                for (int c0 = half * (kAccCols / kGroups); c0 < (half + 1) * (kAccCols / kGroups); c0 += 32) {
-                    uint32_t acc[32];
-                    TMEM_LD32(tmem_o + lane_base + c0, acc, 0);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) acc[c] = __float_as_uint(__uint_as_float(acc[c]) * alpha);
-                    TMEM_ST32(tmem_o + lane_base + c0, acc, 0);
-                }
-            }
-            l_run *= alpha;
-            r_run *= alpha;
+#if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
+                const bool trace_me = trace_on && lane == 0;
+                if (trace_me && g < kTraceSteps) g_trace[5 + (warp - kFirstSoftmaxWarp)][g] = clock64();     // softmax warp: scores seen ready
+#endif
+                const uint32_t tm_s = tmem + lane_base + kScoreCol0 + bsel * kScoreBufStride;
+                const uint32_t tm_ts = tm_s + kBlockN;
 
-            // P~ = exp(S - m_new), l += rowsum(P~)   (two columns per FMA-pipe instruction)
-            const uint64_t c1c1 = pack_f32x2(c1, c1);
-            const uint64_t negm = pack_f32x2(-m_ref, -m_ref);
-            uint64_t ls2[2] = {0ull, 0ull};     // (+0.0f, +0.0f)
+                uint32_t sv[kBlockN];
+                uint32_t tv[kBlockN];
 #pragma unroll
-            for (int c = 0; c < kHalfN; c += 2) {
-                float x0, x1;
-                unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), c1c1, negm), x0, x1);
-                const float p0 = ex2f(x0), p1 = ex2f(x1);
-                sv[c] = __float_as_uint(p0);
-                sv[c + 1] = __float_as_uint(p1);
-                ls2[(c >> 1) & 1] = add_f32x2(ls2[(c >> 1) & 1], pack_f32x2(p0, p1));
-            }
-            float ls4[4];
-            unpack_f32x2(ls2[0], ls4[0], ls4[1]);
-            unpack_f32x2(ls2[1], ls4[2], ls4[3]);
-            if (valid < kHalfN) {
-                // exact zeros for masked keys whatever the scale (0 * inf above would give NaN)
-                ls4[0] = ls4[1] = ls4[2] = ls4[3] = 0.0f;
-#pragma unroll
-                for (int c = 0; c < kHalfN; ++c) {
-                    if (c >= valid) sv[c] = 0u;
-                    ls4[c & 3] += __uint_as_float(sv[c]);
+                for (int c0 = 0; c0 < kBlockN; c0 += 32) {
+                    TMEM_LD32(tm_s + c0, sv, c0);
+                    if (kHasTQ) TMEM_LD32(tm_ts + c0, tv, c0);
                 }
-            }
-            const float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
-            l_run += lsum;
-            {
-                uint32_t pk[kHalfN / 2];
+                tc_wait_ld();
+
+                // keys past Lk (zero-filled by TMA) must not enter the softmax
+                const int valid = args.Lk - (w.tile0 + j) * kBlockN;
+                if (valid < kBlockN) {
+                    const uint32_t masked = neg_scale ? 0x7F800000u : 0xFF800000u;   // -inf after scaling
 #pragma unroll
-                for (int c = 0; c < kHalfN / 2; ++c) pk[c] = pack_bf16(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1]));
+                    for (int c = 0; c < kBlockN; ++c) if (c >= valid) sv[c] = masked;
+                }
+
+                // rowmax(S_ij) (four independent chains), in the log2 domain
+                float mx4[4];
 #pragma unroll
-                for (int c0 = 0; c0 < kHalfN / 2; c0 += 16) TMEM_ST16(tm_s + half * (kHalfN / 2) + c0, pk, c0);
-            }
-            if (kHasTQ) {
-                // tO does not change when a per-row constant is subtracted from tS (softmax is shift
-                // invariant: the constant leaves H~ V - (r/l) O unchanged).  Centring tS on its P-weighted
-                // mean over the first tile keeps H~ and r small, so that the bf16 rounding of H~ scales
-                // with |tS - mu| instead of |tS| when the two terms cancel in the epilogue.
-                if (j == 0) {
-                    float nm4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                for (int u = 0; u < 4; ++u) mx4[u] = __uint_as_float(sv[u]);
+                if (!neg_scale) {
 #pragma unroll
-                    for (int c = 0; c < kHalfN; ++c)
-                        nm4[c & 3] = fmaf(__uint_as_float(sv[c]), __uint_as_float(tv[c]) * sc, nm4[c & 3]);
-                    // The two owners of a row swap their partial sums through tensor memory: columns
-                    // 32.. of the S buffer are dead once both have loaded their scores (the exchange of
-                    // the maxima above guarantees that) and both threads address the same lane.
-                    const float num_h = (nm4[0] + nm4[1]) + (nm4[2] + nm4[3]);
-                    if (kGroups == 2) {
-                        float num_o, lsum_o;
-                        tmem_st2(tm_s + kBlockN / 2 + 2 * half, num_h, lsum);
-                        tc_wait_st();
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(smem_u32(&bar_xchg[2][quarter]));
-                        if (!mbar_wait_warp(smem_u32(&bar_xchg[2][quarter]), 0, abort_state)) { ok = false; break; }
-                        tc_fence_after();
-                        tmem_ld2(tm_s + kBlockN / 2 + 2 * (half ^ 1), num_o, lsum_o);
+                    for (int c = 4; c < kBlockN; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(sv[c]));
+                } else {
+#pragma unroll
+                    for (int c = 4; c < kBlockN; ++c) mx4[c & 3] = fminf(mx4[c & 3], __uint_as_float(sv[c]));
+                }
+                float mx = neg_scale ? fminf(fminf(mx4[0], mx4[1]), fminf(mx4[2], mx4[3]))
+                                     : fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                mx *= c1;
+
+                // m_new = max(m, rowmax), applied lazily: the result does not depend on which
+                // reference is used as long as exp() stays in range.
+                float alpha = 1.0f;
+                const bool need = mx > m_ref + kRescaleThreshold;
+                if (need) {
+                    alpha = ex2f(m_ref - mx);    // e^{m - m_new}; 0 on the first tile (m = -inf)
+                    m_ref = mx;
+                }
+                if (j > 0 && __any_sync(0xffffffffu, need)) {
+                    // the accumulators must be complete up to tile j-1 before they are rescaled
+                    if (!mbar_wait_warp(smem_u32(&bar_pv_done), (g - 1) & 1, abort_state)) { ok = false; break; }
+                    tc_fence_after();
+                    constexpr int kAccCols = kHasTQ ? 2 * D : D;
+#pragma unroll 1
+                    for (int c0 = 0; c0 < kAccCols; c0 += 32) {
+                        uint32_t acc[32];
+                        TMEM_LD32(tmem_o + lane_base + c0, acc, 0);
                         tc_wait_ld();
-                        // same operand order in both threads, so that both get the same bits
-                        ts_shift = half == 0 ? (num_h + num_o) / (lsum + lsum_o) : (num_o + num_h) / (lsum_o + lsum);
-                    } else {
-                        ts_shift = num_h / lsum;
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) acc[c] = __float_as_uint(__uint_as_float(acc[c]) * alpha);
+                        TMEM_ST32(tmem_o + lane_base + c0, acc, 0);
                     }
                 }
-                // H~ = P~ . tS, r += rowsum(H~)
-                const uint64_t scsc = pack_f32x2(sc, sc);
-                const uint64_t negshift = pack_f32x2(-ts_shift, -ts_shift);
-                uint64_t rs2[2] = {0ull, 0ull};
-#pragma unroll
-                for (int c = 0; c < kHalfN; c += 2) {
-                    const uint64_t ts2 = fma_f32x2(pack_f32x2(__uint_as_float(tv[c]), __uint_as_float(tv[c + 1])), scsc, negshift);
-                    const uint64_t h2 = mul_f32x2(pack_f32x2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), ts2);
-                    float h0, h1;
-                    unpack_f32x2(h2, h0, h1);
-                    tv[c] = __float_as_uint(h0);
-                    tv[c + 1] = __float_as_uint(h1);
-                    rs2[(c >> 1) & 1] = add_f32x2(rs2[(c >> 1) & 1], h2);
-                }
-                {
-                    float a0, a1, a2, a3;
-                    unpack_f32x2(rs2[0], a0, a1);
-                    unpack_f32x2(rs2[1], a2, a3);
-                    r_run += (a0 + a1) + (a2 + a3);
-                }
-                uint32_t pk[kHalfN / 2];
-#pragma unroll
-                for (int c = 0; c < kHalfN / 2; ++c) pk[c] = pack_bf16(__uint_as_float(tv[2 * c]), __uint_as_float(tv[2 * c + 1]));
-#pragma unroll
-                for (int c0 = 0; c0 < kHalfN / 2; c0 += 16) TMEM_ST16(tm_ts + half * (kHalfN / 2) + c0, pk, c0);
-            }
-            tc_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bar_p_full[bsel]));
-#if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
-            if (trace_me && j < kTraceSteps) g_trace[13 + (warp - kFirstSoftmaxWarp)][j] = clock64();    // softmax warp: arrived
-#endif
-        }
+                l_run *= alpha;
+                r_run *= alpha;
 
-        // Epilogue: O/l, L = m + log l, tO = (T - r (O/l)) / l
-        // A parity wait can only tell the current phase from the previous one, and the value MMAs of
-        // tile n-2 may still be running here: wait for them first, then for those of tile n-1.
-        if (ok && n_kv >= 2) ok = mbar_wait_warp(smem_u32(&bar_pv_done), (n_kv - 2) & 1, abort_state);
-        if (ok) ok = mbar_wait_warp(smem_u32(&bar_pv_done), (n_kv - 1) & 1, abort_state);
-        if (ok && kGroups == 2) {
-            // total l and r of the row = sum of the two halves' shares, swapped through the (now dead)
-            // score columns of tensor memory.
-            tc_fence_after();
-            const uint32_t tm_x = tmem + lane_base + kScoreCol0 + kBlockN / 2;
-            tmem_st2(tm_x + 2 * half, l_run, r_run);
-            tc_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bar_xchg[2][quarter]));
-            ok = mbar_wait_warp(smem_u32(&bar_xchg[2][quarter]), kHasTQ ? 1 : 0, abort_state);   // phase 0 was the first-tile exchange
-        }
-        if (ok) {
-            tc_fence_after();
-            float l_tot = l_run, r_tot = r_run;
-            if (kGroups == 2) {
-                float l_o, r_o;
-                tmem_ld2(tmem + lane_base + kScoreCol0 + kBlockN / 2 + 2 * (half ^ 1), l_o, r_o);
-                tc_wait_ld();
-                l_tot = half == 0 ? l_run + l_o : l_o + l_run;
-                r_tot = half == 0 ? r_run + r_o : r_o + r_run;
+                // P~ = exp(S - m_new), l += rowsum(P~)   (two columns per FMA-pipe instruction)
+                const uint64_t c1c1 = pack_f32x2(c1, c1);
+                const uint64_t negm = pack_f32x2(-m_ref, -m_ref);
+                uint64_t ls2[2] = {0ull, 0ull};     // (+0.0f, +0.0f)
+#pragma unroll
+                for (int c = 0; c < kBlockN; c += 2) {
+                    float x0, x1;
+                    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), c1c1, negm), x0, x1);
+                    const float p0 = ex2f(x0), p1 = ex2f(x1);
+                    sv[c] = __float_as_uint(p0);
+                    sv[c + 1] = __float_as_uint(p1);
+                    ls2[(c >> 1) & 1] = add_f32x2(ls2[(c >> 1) & 1], pack_f32x2(p0, p1));
+                }
+                float ls4[4];
+                unpack_f32x2(ls2[0], ls4[0], ls4[1]);
+                unpack_f32x2(ls2[1], ls4[2], ls4[3]);
+                if (valid < kBlockN) {
+                    // exact zeros for masked keys whatever the scale (0 * inf above would give NaN)
+                    ls4[0] = ls4[1] = ls4[2] = ls4[3] = 0.0f;
+#pragma unroll
+                    for (int c = 0; c < kBlockN; ++c) {
+                        if (c >= valid) sv[c] = 0u;
+                        ls4[c & 3] += __uint_as_float(sv[c]);
+                    }
+                }
+                const float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+                l_run += lsum;
+                {
+                    uint32_t pk[kBlockN / 2];
+#pragma unroll
+                    for (int c = 0; c < kBlockN / 2; ++c) pk[c] = pack_bf16(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1]));
+                    TMEM_ST32(tm_s, pk, 0);
+                }
+                if (kHasTQ) {
+                    // tO does not change when a per-row constant is subtracted from tS (softmax is shift
+                    // invariant: the constant leaves H~ V - (r/l) O unchanged).  Centring tS on its P-weighted
+                    // mean over the first tile keeps H~ and r small, so that the bf16 rounding of H~ scales
+                    // with |tS - mu| instead of |tS| when the two terms cancel in the epilogue.
+                    if (j == 0) {
+                        float nm4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+                        for (int c = 0; c < kBlockN; ++c)
+                            nm4[c & 3] = fmaf(__uint_as_float(sv[c]), __uint_as_float(tv[c]) * sc, nm4[c & 3]);
+                        ts_shift = ((nm4[0] + nm4[1]) + (nm4[2] + nm4[3])) / lsum;
+                    }
+                    // H~ = P~ . tS, r += rowsum(H~)
+                    const uint64_t scsc = pack_f32x2(sc, sc);
+                    const uint64_t negshift = pack_f32x2(-ts_shift, -ts_shift);
+                    uint64_t rs2[2] = {0ull, 0ull};
+#pragma unroll
+                    for (int c = 0; c < kBlockN; c += 2) {
+                        const uint64_t ts2 = fma_f32x2(pack_f32x2(__uint_as_float(tv[c]), __uint_as_float(tv[c + 1])), scsc, negshift);
+                        const uint64_t h2 = mul_f32x2(pack_f32x2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), ts2);
+                        float h0, h1;
+                        unpack_f32x2(h2, h0, h1);
+                        tv[c] = __float_as_uint(h0);
+                        tv[c + 1] = __float_as_uint(h1);
+                        rs2[(c >> 1) & 1] = add_f32x2(rs2[(c >> 1) & 1], h2);
+                    }
+                    {
+                        float a0, a1, a2, a3;
+                        unpack_f32x2(rs2[0], a0, a1);
+                        unpack_f32x2(rs2[1], a2, a3);
+                        r_run += (a0 + a1) + (a2 + a3);
+                    }
+                    uint32_t pk[kBlockN / 2];
+#pragma unroll
+                    for (int c = 0; c < kBlockN / 2; ++c) pk[c] = pack_bf16(__uint_as_float(tv[2 * c]), __uint_as_float(tv[2 * c + 1]));
+                    TMEM_ST32(tm_ts, pk, 0);
+                }
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bar_p_full[bsel]));
+#if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
+                if (trace_me && g < kTraceSteps) g_trace[13 + (warp - kFirstSoftmaxWarp)][g] = clock64();    // softmax warp: arrived
+#endif
             }
-            const int qi = q0 + row;
+            if (!ok) break;
+
+            // Epilogue: O/l, L = m + log l, tO = (T - r (O/l)) / l
+            // A parity wait can only tell the current phase from the previous one, and the value MMAs of
+            // tile n-2 may still be running here: wait for them first, then for those of tile n-1.
+            const int g_last = g0 + n_kv - 1;
+            if (n_kv >= 2) ok = mbar_wait_warp(smem_u32(&bar_pv_done), (g_last - 1) & 1, abort_state);
+            if (ok) ok = mbar_wait_warp(smem_u32(&bar_pv_done), g_last & 1, abort_state);
+            if (!ok) break;
+            tc_fence_after();
+            const float l_tot = l_run, r_tot = r_run;
+            const int qi = w.q0 + row;
             const bool in_range = qi < args.Lq;
             const float inv_l = 1.0f / l_tot;
             const float mu = r_tot * inv_l;
+            const int b = w.b, h = w.h, split = w.split;
             const size_t row_off = ((static_cast<size_t>(b) * args.Lq + (in_range ? qi : 0)) * args.H + h) * D;
             // split-KV: this chunk's normalised partial results go to the fp32 scratch of chunk `split`
             const size_t part_off = kSplit ? static_cast<size_t>(split) * args.B * args.Lq * args.H * D + row_off : 0;
@@ -929,12 +912,18 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             float* po_row = kSplit ? args.part_o + part_off : nullptr;
             float* pto_row = (kSplit && kHasTQ) ? args.part_to + part_off : nullptr;
 #pragma unroll 1
-            for (int c0 = half * (D / kGroups); c0 < (half + 1) * (D / kGroups); c0 += 32) {
+            for (int c0 = 0; c0 < D; c0 += 32) {
                 uint32_t ov[32];
                 uint32_t tvv[32];
                 TMEM_LD32(tmem_o + lane_base + c0, ov, 0);
                 if (kHasTQ) TMEM_LD32(tmem_t + lane_base + c0, tvv, 0);
                 tc_wait_ld();
+                if (c0 + 32 >= D) {
+                    // O and T are in registers: the next item's first value MMA may overwrite them
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bar_acc_free));
+                }
                 if (kSplit) {
 #pragma unroll
                     for (int c = 0; c < 32; ++c) {
@@ -973,7 +962,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     }
                 }
             }
-            if (in_range && half == 0) {
+            if (in_range) {
                 // L = m + log l (natural log); mu = r / l, plus the constant that was taken out of tS
                 const float lse_val = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
                 const float mu_val = kHasTQ ? mu + ts_shift : 0.0f;
@@ -987,6 +976,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (args.mu != nullptr) args.mu[idx] = mu_val;
                 }
             }
+            g0 += n_kv;
         }
     }
 
