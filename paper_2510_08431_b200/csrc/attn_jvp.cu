@@ -99,7 +99,8 @@ int launch(const CUtensorMap* maps, const KernelArgs& ka, dim3 grid, cudaStream_
         if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
         smem = want;
     }
-    kern<<<grid, attn_jvp::kThreads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], ka);
+    kern<<<grid, attn_jvp::kThreads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], maps[6],
+                                                     maps[7], ka);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail("kernel launch", e);
     return 0;
@@ -195,13 +196,16 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     }
 
     // ---- tensor maps (Q-side boxes are 128 rows, K-side boxes 64 rows) ----
-    CUtensorMap maps[6];
+    CUtensorMap maps[8];
     if (int rc = make_map(&maps[0], q, B, Lq, H, D, attn_jvp::kBlockM)) return rc;
     if (int rc = make_map(&maps[1], k, B, Lk, H, D, attn_jvp::kBlockN)) return rc;
     if (int rc = make_map(&maps[2], v, B, Lk, H, D, attn_jvp::kBlockN)) return rc;
     if (int rc = make_map(&maps[3], fwd_only ? q : tq, B, Lq, H, D, attn_jvp::kBlockM)) return rc;
     if (int rc = make_map(&maps[4], mode == attn_jvp::kModeJvp ? tk : k, B, Lk, H, D, attn_jvp::kBlockN)) return rc;
     if (int rc = make_map(&maps[5], mode == attn_jvp::kModeJvp ? tv : v, B, Lk, H, D, attn_jvp::kBlockN)) return rc;
+    // output tiles (bf16, stored from shared memory by TMA; the split-KV kernel does not use these two)
+    if (int rc = make_map(&maps[6], o, B, Lq, H, D, attn_jvp::kBlockM)) return rc;
+    if (int rc = make_map(&maps[7], fwd_only ? o : to, B, Lq, H, D, attn_jvp::kBlockM)) return rc;
 
     KernelArgs ka;
     ka.o = reinterpret_cast<__nv_bfloat16*>(o);

@@ -189,6 +189,23 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
+// Tile store shared -> global through a tensor map (rows beyond the tensor's extent are clipped).
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+        ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// The stores committed so far have read their shared-memory source (it may be overwritten).
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// The stores committed so far are complete.
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// Orders this thread's shared-memory writes before later reads by the asynchronous proxy (TMA).
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
@@ -341,12 +358,18 @@ __global__ void __launch_bounds__(kThreads, 1)
 attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_tq,
                     const __grid_constant__ CUtensorMap tm_tk, const __grid_constant__ CUtensorMap tm_tv,
+                    const __grid_constant__ CUtensorMap tm_o, const __grid_constant__ CUtensorMap tm_to,
                     const KernelArgs args) {
     using Plan = SmemPlan<D>;
     constexpr int kHalves = Plan::kHalves;
     constexpr int kSlots = Plan::kSlots;
     constexpr bool kHasTQ = (MODE != kModeFwdOnly);          // tS and T exist
     constexpr bool kHasTKV = (MODE == kModeJvp);             // tK, tV are read
+    // The bf16 output tiles leave through shared memory and TMA stores: at the end of every item the ring gives
+    // up one slot per output tensor (a slot is exactly one 128 x D bf16 tile).  The split-KV kernel writes its
+    // fp32 partial results straight from registers and stages nothing.
+    constexpr int kStageSlots = kSplit ? 0 : (kHasTQ ? 2 : 1);
+    static_assert(Plan::kSlotBytes == Plan::kQBytes, "an output tile must fill one ring slot");
 
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_q_full;     // Q, tQ of the current work item are in shared memory
@@ -358,6 +381,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     __shared__ __align__(8) uint64_t bar_pv_done;
     __shared__ __align__(8) uint64_t bar_acc_free;   // the epilogue has read O and T: the next item may overwrite them
     __shared__ __align__(8) uint64_t bar_drain;
+    __shared__ __align__(8) uint64_t bar_stage_ready;   // the item's staging slots are free of operand reads
+    __shared__ __align__(8) uint64_t bar_stage_full;    // the softmax warps have written the item's output tiles
     __shared__ uint32_t tmem_base_smem;
     __shared__ int cta_abort;
 
@@ -426,6 +451,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         mbar_init(smem_u32(&bar_pv_done), 1);
         mbar_init(smem_u32(&bar_acc_free), kSoftmaxThreads / 32);
         mbar_init(smem_u32(&bar_drain), 1);
+        mbar_init(smem_u32(&bar_stage_ready), 1);
+        mbar_init(smem_u32(&bar_stage_full), kSoftmaxThreads / 32);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kMmaWarp) {
@@ -439,6 +466,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         prefetch_tensormap(&tm_v);
         if (kHasTQ) prefetch_tensormap(&tm_tq);
         if (kHasTKV) { prefetch_tensormap(&tm_tk); prefetch_tensormap(&tm_tv); }
+        if (kStageSlots > 0) prefetch_tensormap(&tm_o);
+        if (kStageSlots > 1) prefetch_tensormap(&tm_to);
     }
     tc_fence_before();
     __syncthreads();
@@ -449,7 +478,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
     // Phases.  Key tiles are numbered g = 0, 1, 2, ... over ALL items of this CTA; tile g uses score buffer g & 1,
     // phase (g >> 1) & 1 of bar_s_full / bar_p_full and phase g & 1 of bar_pv_done.  Item number `it` (0, 1, ...)
-    // uses phase it & 1 of bar_q_full / bar_q_free / bar_acc_free.  The shared-memory ring runs on without a break.
+    // uses phase it & 1 of bar_q_full / bar_q_free / bar_acc_free / bar_stage_ready / bar_stage_full.  The
+    // shared-memory ring runs on without a break; per item it hands out 2 n slots to K/V tiles and then
+    // kStageSlots slots to the output tiles.
 
     if (warp == kProducerWarp) {
         // =====================================================================================
@@ -461,23 +492,29 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             constexpr uint32_t kKTx = (kHasTKV ? 2u : 1u) * kHalves * Plan::kKvHalfBytes;
             constexpr uint32_t kVTx = kKTx;
             const uint32_t qbar = smem_u32(&bar_q_full);
-            int t = 0;          // ring position
+            // ring position: slot, the parity of the slot's `full` phase that this lap completes, and whether the
+            // ring has been round once (before that the slots are empty without anybody saying so)
+            int r_slot = 0;
+            uint32_t r_parity = 0;
+            bool r_lapped = false;
             bool ok = true;
             Item w{};
-            auto acquire = [&](uint32_t& slot_addr, uint32_t& bar) -> bool {
-                const int slot = t % kSlots;
-                if (t >= kSlots) {
-                    if (!mbar_wait(smem_u32(&bar_slot_empty[slot]), ((t / kSlots) - 1) & 1, abort_state)) return false;
+            // waits until the slot at the ring position is empty, hands it out and moves on
+            auto acquire = [&](int& slot, uint32_t& slot_addr, uint32_t& bar) -> bool {
+                slot = r_slot;
+                if (r_lapped) {
+                    if (!mbar_wait(smem_u32(&bar_slot_empty[slot]), r_parity ^ 1u, abort_state)) return false;
                 }
                 slot_addr = smem_ring + slot * Plan::kSlotBytes;
                 bar = smem_u32(&bar_slot_full[slot]);
-                TRACE(0, t);          // producer: slot t acquired, loads issued next
-                ++t;
+                TRACE(0, slot);       // producer: slot acquired, loads issued next
+                if (++r_slot == kSlots) { r_slot = 0; r_parity ^= 1u; r_lapped = true; }
                 return true;
             };
             auto load_k = [&](int j) -> bool {
+                int slot;
                 uint32_t dst, bar;
-                if (!acquire(dst, bar)) return false;
+                if (!acquire(slot, dst, bar)) return false;
                 mbar_arrive_expect_tx(bar, kKTx);
                 // per 64-column half: [K_half (8 KB)][tK_half (8 KB)] so that [K ; tK] is one N = 128 operand
 #pragma unroll
@@ -489,8 +526,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 return true;
             };
             auto load_v = [&](int j) -> bool {
+                int slot;
                 uint32_t dst, bar;
-                if (!acquire(dst, bar)) return false;
+                if (!acquire(slot, dst, bar)) return false;
                 mbar_arrive_expect_tx(bar, kVTx);
                 // [V_half0][V_half1][tV_half0][tV_half1]: consecutive 64-wide N atoms of [V | tV]
 #pragma unroll
@@ -499,6 +537,28 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (kHasTKV)
                         tma_load_4d(dst + (kHalves + hf) * Plan::kKvHalfBytes, &tm_tv, bar, hf * 64, w.h, (w.tile0 + j) * kBlockN, w.b);
                 }
+                return true;
+            };
+            // Output tiles of the item before: staged by the softmax warps in `stage_slot[]`, stored from here.
+            bool stage_pending = false;
+            int stage_slot[2] = {0, 0};
+            int stage_it = 0;
+            Item stage_w{};
+            auto store_staged = [&]() -> bool {
+                if (!mbar_wait(smem_u32(&bar_stage_full), stage_it & 1, abort_state)) return false;
+#pragma unroll
+                for (int hf = 0; hf < kHalves; ++hf) {
+                    tma_store_4d(&tm_o, smem_ring + stage_slot[0] * Plan::kSlotBytes + hf * Plan::kQHalfBytes,
+                                 hf * 64, stage_w.h, stage_w.q0, stage_w.b);
+                    if (kStageSlots > 1)
+                        tma_store_4d(&tm_to, smem_ring + stage_slot[1] * Plan::kSlotBytes + hf * Plan::kQHalfBytes,
+                                     hf * 64, stage_w.h, stage_w.q0, stage_w.b);
+                }
+                tma_store_commit();
+                tma_store_wait_read();
+                // the slots go back to the ring (their `empty` phase is completed here instead of by an MMA commit)
+                for (int s = 0; s < kStageSlots; ++s) mbar_arrive(smem_u32(&bar_slot_empty[stage_slot[s]]));
+                stage_pending = false;
                 return true;
             };
             int it = 0;
@@ -516,14 +576,38 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 for (int j = 0; ok && j < w.n_kv; ++j) {
                     if (j + 1 < w.n_kv) ok = load_k(j + 1);
                     if (ok) ok = load_v(j);
+                    // the previous item's outputs, once this item's first loads are on their way
+                    if (ok && j == 0 && stage_pending) ok = store_staged();
+                }
+                if (kStageSlots > 0 && ok) {
+                    // hand the item's staging slots to the softmax warps; nothing is loaded into them, so their
+                    // `full` phase is completed by a plain arrival to keep the ring's parities in step
+                    for (int s = 0; ok && s < kStageSlots; ++s) {
+                        uint32_t dst, bar;
+                        ok = acquire(stage_slot[s], dst, bar);
+                        if (ok) mbar_arrive(bar);
+                    }
+                    if (ok) {
+                        mbar_arrive(smem_u32(&bar_stage_ready));
+                        stage_pending = true;
+                        stage_it = it;
+                        stage_w = w;
+                    }
                 }
             }
+            if (ok && stage_pending) ok = store_staged();
+            if (kStageSlots > 0) tma_store_wait_all();
             if (!ok) {
                 // Abandoning the work: let the copies already in flight land before the CTA exits.
-                const int issued = t;
-                for (int u = (issued > kSlots ? issued - kSlots : 0); u < issued; ++u) {
-                    const uint32_t bar = smem_u32(&bar_slot_full[u % kSlots]);
-                    const uint32_t par = (u / kSlots) & 1;
+                // Walk back over the last positions handed out (at most one lap): each slot's current `full`
+                // phase completes when its copy has landed (or at once, for a staging slot).
+                const int back = r_lapped ? kSlots : r_slot;
+                int slot = r_slot;
+                uint32_t par = r_parity;
+                for (int u = 0; u < back; ++u) {
+                    if (slot == 0) { slot = kSlots; par ^= 1u; }
+                    --slot;
+                    const uint32_t bar = smem_u32(&bar_slot_full[slot]);
                     const unsigned long long t0 = globaltimer_ns();
                     while (!mbar_try_wait(bar, par) && globaltimer_ns() - t0 < 100000000ull) {}
                 }
@@ -708,6 +792,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     has_k = nxt_has_k;
                 }
                 g0 += n_kv;
+                // the ring positions after the item's last V tile belong to the output staging
+                for (int s = 0; s < kStageSlots; ++s) advance(pos);
             }
             if (!ok && leader) {
                 // Abandoning the work: wait (bounded) until the tensor core has drained what was issued.
@@ -731,6 +817,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         bool ok = true;
         int g0 = 0;          // global number of the item's first key tile
         int it = 0;
+        int ring_slot = 0;   // ring slot of the item's first position (the ring hands out 2 n + kStageSlots per item)
 
         for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
             const Item w = decode(item);
@@ -907,10 +994,19 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             const size_t row_off = ((static_cast<size_t>(b) * args.Lq + (in_range ? qi : 0)) * args.H + h) * D;
             // split-KV: this chunk's normalised partial results go to the fp32 scratch of chunk `split`
             const size_t part_off = kSplit ? static_cast<size_t>(split) * args.B * args.Lq * args.H * D + row_off : 0;
-            __nv_bfloat16* o_row = args.o + row_off;
-            __nv_bfloat16* to_row = kHasTQ ? args.to + row_off : nullptr;
             float* po_row = kSplit ? args.part_o + part_off : nullptr;
             float* pto_row = (kSplit && kHasTQ) ? args.part_to + part_off : nullptr;
+            // bf16 outputs: staged in the ring slots after the item's last V tile, in the 128-byte-swizzled
+            // layout of the output tensor maps (row r, 16-byte chunk c of a 64-column half at r*128 + (c ^ (r&7))*16)
+            uint32_t stage_o = 0, stage_t = 0;
+            if (kStageSlots > 0) {
+                const int so = (ring_slot + 2 * (n_kv % kSlots)) % kSlots;
+                stage_o = smem_ring + so * Plan::kSlotBytes + row * 128;
+                stage_t = smem_ring + ((so + 1) % kSlots) * Plan::kSlotBytes + row * 128;
+                ring_slot = (so + kStageSlots) % kSlots;
+                ok = mbar_wait_warp(smem_u32(&bar_stage_ready), it & 1, abort_state);
+                if (!ok) break;
+            }
 #pragma unroll 1
             for (int c0 = 0; c0 < D; c0 += 32) {
                 uint32_t ov[32];
@@ -952,15 +1048,22 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                             pt[c] = pack_bf16(t0, t1);
                         }
                     }
-                    if (in_range) {
+                    // rows beyond Lq are staged too (the store clips them)
+                    const uint32_t half_off = (c0 >> 6) * Plan::kQHalfBytes;
+                    const int chunk0 = (c0 & 63) >> 3;
 #pragma unroll
-                        for (int v4 = 0; v4 < 4; ++v4) {
-                            *reinterpret_cast<uint4*>(o_row + c0 + v4 * 8) = make_uint4(po[4 * v4], po[4 * v4 + 1], po[4 * v4 + 2], po[4 * v4 + 3]);
-                            if (kHasTQ)
-                                *reinterpret_cast<uint4*>(to_row + c0 + v4 * 8) = make_uint4(pt[4 * v4], pt[4 * v4 + 1], pt[4 * v4 + 2], pt[4 * v4 + 3]);
-                        }
+                    for (int v4 = 0; v4 < 4; ++v4) {
+                        const uint32_t off = half_off + (((chunk0 + v4) ^ (row & 7)) << 4);
+                        st_shared_v4(stage_o + off, po[4 * v4], po[4 * v4 + 1], po[4 * v4 + 2], po[4 * v4 + 3]);
+                        if (kHasTQ) st_shared_v4(stage_t + off, pt[4 * v4], pt[4 * v4 + 1], pt[4 * v4 + 2], pt[4 * v4 + 3]);
                     }
                 }
+            }
+            if (kStageSlots > 0) {
+                // the staged tiles are complete: the producer thread stores them
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bar_stage_full));
             }
             if (in_range) {
                 // L = m + log l (natural log); mu = r / l, plus the constant that was taken out of tS
