@@ -206,6 +206,11 @@ __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.b
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // Orders this thread's shared-memory writes before later reads by the asynchronous proxy (TMA).
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// Brings a tile into L2 only.
+__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap* map, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
@@ -546,6 +551,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             Item stage_w{};
             auto store_staged = [&]() -> bool {
                 if (!mbar_wait(smem_u32(&bar_stage_full), stage_it & 1, abort_state)) return false;
+                TRACE(17, stage_it);  // producer: staged tiles complete, stores issued next
 #pragma unroll
                 for (int hf = 0; hf < kHalves; ++hf) {
                     tma_store_4d(&tm_o, smem_ring + stage_slot[0] * Plan::kSlotBytes + hf * Plan::kQHalfBytes,
@@ -558,42 +564,63 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 tma_store_wait_read();
                 // the slots go back to the ring (their `empty` phase is completed here instead of by an MMA commit)
                 for (int s = 0; s < kStageSlots; ++s) mbar_arrive(smem_u32(&bar_slot_empty[stage_slot[s]]));
+                TRACE(18, stage_it);  // producer: staging slots back in the ring
                 stage_pending = false;
                 return true;
             };
+            // hands the staging slots of item number `of_it` to the softmax warps; nothing is loaded into them, so
+            // their `full` phase is completed by a plain arrival to keep the ring's parities in step
+            auto acquire_stage = [&](int of_it, const Item& of_w) -> bool {
+                for (int s = 0; s < kStageSlots; ++s) {
+                    uint32_t dst, bar;
+                    if (!acquire(stage_slot[s], dst, bar)) return false;
+                    mbar_arrive(bar);
+                }
+                mbar_arrive(smem_u32(&bar_stage_ready));
+                TRACE(9, of_it);      // producer: staging slots handed over
+                stage_pending = true;
+                stage_it = of_it;
+                stage_w = of_w;
+                return true;
+            };
+            Item prev_w{};
             int it = 0;
             for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
                 w = decode(item);
                 if (it > 0) ok = mbar_wait(smem_u32(&bar_q_free), (it - 1) & 1, abort_state);
                 if (!ok) break;
+                TRACE(1, it);         // producer: Q, tQ may be replaced
                 mbar_arrive_expect_tx(qbar, kQTx);
 #pragma unroll
                 for (int hf = 0; hf < kHalves; ++hf) {
                     tma_load_4d(smem_q + hf * Plan::kQHalfBytes, &tm_q, qbar, hf * 64, w.h, w.q0, w.b);
                     if (kHasTQ) tma_load_4d(smem_tq + hf * Plan::kQHalfBytes, &tm_tq, qbar, hf * 64, w.h, w.q0, w.b);
                 }
+                const bool has_next = n_items - item > static_cast<int>(gridDim.x);
+                if (has_next) {
+                    // the next item's Q, tQ can only be loaded once this item's score MMAs are done: have them
+                    // waiting in L2 by then
+                    const Item nx = decode(item + gridDim.x);
+#pragma unroll
+                    for (int hf = 0; hf < kHalves; ++hf) {
+                        tma_prefetch_4d(&tm_q, hf * 64, nx.h, nx.q0, nx.b);
+                        if (kHasTQ) tma_prefetch_4d(&tm_tq, hf * 64, nx.h, nx.q0, nx.b);
+                    }
+                }
                 ok = load_k(0);
+                if (ok && w.n_kv > 1) ok = load_k(1);
+                // staging slots of the item before: after this item's leading K tiles (which the first score MMAs
+                // need at once) and before its V tiles (which are not needed until the first softmax is through)
+                if (kStageSlots > 0 && ok && it > 0) ok = acquire_stage(it - 1, prev_w);
                 for (int j = 0; ok && j < w.n_kv; ++j) {
-                    if (j + 1 < w.n_kv) ok = load_k(j + 1);
+                    if (j >= 1 && j + 1 < w.n_kv) ok = load_k(j + 1);
                     if (ok) ok = load_v(j);
-                    // the previous item's outputs, once this item's first loads are on their way
-                    if (ok && j == 0 && stage_pending) ok = store_staged();
+                    // the previous item's outputs: the loads above do not depend on its epilogue, the later ones do
+                    if (ok && stage_pending && (j == 1 || j + 1 == w.n_kv)) ok = store_staged();
                 }
-                if (kStageSlots > 0 && ok) {
-                    // hand the item's staging slots to the softmax warps; nothing is loaded into them, so their
-                    // `full` phase is completed by a plain arrival to keep the ring's parities in step
-                    for (int s = 0; ok && s < kStageSlots; ++s) {
-                        uint32_t dst, bar;
-                        ok = acquire(stage_slot[s], dst, bar);
-                        if (ok) mbar_arrive(bar);
-                    }
-                    if (ok) {
-                        mbar_arrive(smem_u32(&bar_stage_ready));
-                        stage_pending = true;
-                        stage_it = it;
-                        stage_w = w;
-                    }
-                }
+                prev_w = w;
+                // the CTA's last item: its staging slots follow its last V tile
+                if (kStageSlots > 0 && ok && !has_next) ok = acquire_stage(it, w);
             }
             if (ok && stage_pending) ok = store_staged();
             if (kStageSlots > 0) tma_store_wait_all();
@@ -732,8 +759,10 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const Item w = decode(item);
                 const int n_kv = w.n_kv;
                 ok = mbar_wait_warp(smem_u32(&bar_q_full), it & 1, abort_state);
+                if (leader) TRACE(10, it);    // MMA: Q, tQ of the item seen
                 if (ok) ok = wait_full(pos);
                 if (!ok) break;
+                if (leader) TRACE(11, it);    // MMA: K(0) of the item seen
                 tc_fence_after();
                 prepare_k(pos.slot);
                 if (leader) { issue_scores_a(g0); issue_scores_b(g0, pos.slot, n_kv == 1); }
@@ -747,6 +776,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     __syncwarp();
                     advance(pos);
                 }
+                // the ring positions between the item's leading K tiles and V(0) stage the previous item's outputs
+                if (it > 0) { for (int s = 0; s < kStageSlots; ++s) advance(pos); }
                 // pos = V(0).  Per tile j: burst = value MMAs of tile j, score MMAs of tile j+2; the barriers of
                 // tile j+1 are tested in the middle of the burst, while the queue is still full.
                 RingPos pos_v = pos, pos_k = pos;
@@ -792,8 +823,6 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     has_k = nxt_has_k;
                 }
                 g0 += n_kv;
-                // the ring positions after the item's last V tile belong to the output staging
-                for (int s = 0; s < kStageSlots; ++s) advance(pos);
             }
             if (!ok && leader) {
                 // Abandoning the work: wait (bounded) until the tensor core has drained what was issued.
@@ -834,7 +863,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 tc_fence_after();
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
                 const bool trace_me = trace_on && lane == 0;
-                if (trace_me && g < kTraceSteps) g_trace[5 + (warp - kFirstSoftmaxWarp)][g] = clock64();     // softmax warp: scores seen ready
+                if (trace_me && g < kTraceSteps) g_trace[5 + ((warp - kFirstSoftmaxWarp) & 3)][g] = clock64();     // softmax warp: scores seen ready
 #endif
                 const uint32_t tm_s = tmem + lane_base + kScoreCol0 + bsel * kScoreBufStride;
                 const uint32_t tm_ts = tm_s + kBlockN;
@@ -972,7 +1001,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bar_p_full[bsel]));
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
-                if (trace_me && g < kTraceSteps) g_trace[13 + (warp - kFirstSoftmaxWarp)][g] = clock64();    // softmax warp: arrived
+                if (trace_me && g < kTraceSteps) g_trace[13 + ((warp - kFirstSoftmaxWarp) & 3)][g] = clock64();    // softmax warp: arrived
 #endif
             }
             if (!ok) break;
@@ -985,6 +1014,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             if (ok) ok = mbar_wait_warp(smem_u32(&bar_pv_done), g_last & 1, abort_state);
             if (!ok) break;
             tc_fence_after();
+#if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
+            if (trace_on && lane == 0 && ((warp - kFirstSoftmaxWarp) & 3) == 0 && it < kTraceSteps) g_trace[12][it] = clock64();    // softmax warp: epilogue begins
+#endif
             const float l_tot = l_run, r_tot = r_run;
             const int qi = w.q0 + row;
             const bool in_range = qi < args.Lq;
@@ -1000,12 +1032,15 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // layout of the output tensor maps (row r, 16-byte chunk c of a 64-column half at r*128 + (c ^ (r&7))*16)
             uint32_t stage_o = 0, stage_t = 0;
             if (kStageSlots > 0) {
-                const int so = (ring_slot + 2 * (n_kv % kSlots)) % kSlots;
+                // Ring positions of this item: 2 n_kv tiles, plus the previous item's staging slots.  Its own staging
+                // slots come after the next item's leading K tiles (every item has n_kv tiles here: the kernel that
+                // cuts the keys into chunks stages nothing), or right after its last V tile if it is the CTA's last.
+                const bool has_next = n_items - item > static_cast<int>(gridDim.x);
+                const int next_start = (ring_slot + 2 * (n_kv % kSlots) + (it > 0 ? kStageSlots : 0)) % kSlots;
+                const int so = has_next ? (next_start + min(2, n_kv)) % kSlots : next_start;
                 stage_o = smem_ring + so * Plan::kSlotBytes + row * 128;
                 stage_t = smem_ring + ((so + 1) % kSlots) * Plan::kSlotBytes + row * 128;
-                ring_slot = (so + kStageSlots) % kSlots;
-                ok = mbar_wait_warp(smem_u32(&bar_stage_ready), it & 1, abort_state);
-                if (!ok) break;
+                ring_slot = next_start;
             }
 #pragma unroll 1
             for (int c0 = 0; c0 < D; c0 += 32) {
@@ -1013,6 +1048,10 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 uint32_t tvv[32];
                 TMEM_LD32(tmem_o + lane_base + c0, ov, 0);
                 if (kHasTQ) TMEM_LD32(tmem_t + lane_base + c0, tvv, 0);
+                if (kStageSlots > 0 && c0 == 0) {
+                    ok = mbar_wait_warp(smem_u32(&bar_stage_ready), it & 1, abort_state);
+                    if (!ok) { tc_wait_ld(); break; }
+                }
                 tc_wait_ld();
                 if (c0 + 32 >= D) {
                     // O and T are in registers: the next item's first value MMA may overwrite them
@@ -1059,12 +1098,16 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     }
                 }
             }
+            if (!ok) break;
             if (kStageSlots > 0) {
                 // the staged tiles are complete: the producer thread stores them
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bar_stage_full));
             }
+#if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
+            if (trace_on && lane == 0 && ((warp - kFirstSoftmaxWarp) & 3) == 0 && it < kTraceSteps) g_trace[20][it] = clock64();    // softmax warp: epilogue ends
+#endif
             if (in_range) {
                 // L = m + log l (natural log); mu = r / l, plus the constant that was taken out of tS
                 const float lse_val = (m_ref + log2f(l_tot)) * 0.6931471805599453f;
