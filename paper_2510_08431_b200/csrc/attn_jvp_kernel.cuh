@@ -609,6 +609,13 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
                 ok = load_k(0);
                 if (ok && w.n_kv > 1) ok = load_k(1);
+#if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 3
+                {   // timing experiment: when do Q, tQ land?
+                    const unsigned long long t0 = globaltimer_ns();
+                    while (!mbar_test_wait(qbar, it & 1) && globaltimer_ns() - t0 < 1000000ull) {}
+                    TRACE(19, it);
+                }
+#endif
                 // staging slots of the item before: after this item's leading K tiles (which the first score MMAs
                 // need at once) and before its V tiles (which are not needed until the first softmax is through)
                 if (kStageSlots > 0 && ok && it > 0) ok = acquire_stage(it - 1, prev_w);
