@@ -41,7 +41,7 @@ DATASHEET_BF16_TFLOPS = 2250.0
 # DRAM bytes per launch of attn_jvp_fwd_kernel<128, jvp> measured with ncu (dram__bytes_read.sum +
 # dram__bytes_write.sum) on the image_dit_2b workload, see profiles/; scaled to other workloads by their
 # algorithmic bytes (traffic is proportional to the tensors streamed once from HBM; K/V re-reads hit L2).
-NCU_TRAFFIC_BYTES = {"workload": "image_dit_2b", "bytes": 247.9e6}   # 201.5 MB read + 46.5 MB written
+NCU_TRAFFIC_BYTES = {"workload": "image_dit_2b", "bytes": 250.1e6}   # 203.0 MB read + 47.1 MB written (mean of two launches)
 
 
 def algorithmic_bytes(w) -> int:
