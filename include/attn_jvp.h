@@ -60,7 +60,7 @@ extern "C" {
 #define ATTN_JVP_ERR_CUDA            9  /* a CUDA runtime / driver call failed (see strerror) */
 #define ATTN_JVP_ERR_DEVICE_TIMEOUT 10  /* a bounded device-side wait expired */
 #define ATTN_JVP_ERR_DEVICE_LAYOUT  11  /* the kernel's shared-memory layout did not fit (reported like a timeout) */
-#define ATTN_JVP_ERR_WORKSPACE      12  /* split-KV workspace too small */
+#define ATTN_JVP_ERR_WORKSPACE      12  /* the caller's workspace is too small */
 #define ATTN_JVP_ERR_STATIC_SCRATCH 13  /* the call needs more scratch than ATTN_JVP_STATIC_SCRATCH_BYTES */
 
 /* Size of the scratch buffer built into the library for attn_jvp_fwd_splitkv_static (32 MiB). */
@@ -123,6 +123,38 @@ int attn_jvp_fwd_splitkv(const void* q, const void* k, const void* v,
                          int B, int H, int Lq, int Lk, int D,
                          float scale, unsigned flags, int splits,
                          void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * attn_jvp_fwd_host -- the operation of attn_jvp_fwd_stream (Appendix C.1 / Algorithm 2) on HOST tensors.
+ *
+ * q, k, v, tq, tk, tv, o, to, lse are HOST pointers with the layouts of attn_jvp_fwd (bf16 [B][L][H][D], LSE fp32
+ * [B][H][Lq]); page-locked (pinned) memory is needed for the copies to overlap with the kernel, pageable memory
+ * works but is copied synchronously.  The heads are processed in groups of `heads_per_stage`: the group's heads
+ * are gathered out of the interleaved host rows into a dense device copy ([B][L][heads][D]), the kernel runs on
+ * that copy, and its O, tO, LSE are scattered back to the host tensors, while the copy engines already move the
+ * next group in and the previous group out.  Every (b, h) is computed exactly as by attn_jvp_fwd on a device
+ * tensor (the result of a head does not depend on the other heads), so the outputs are bit-identical.
+ *
+ *   heads_per_stage  heads per pipeline stage; 0 = library default (about five stages, copy rows >= 512 bytes).
+ *   workspace        DEVICE scratch owned by the caller, 256-byte aligned, at least
+ *                    attn_jvp_host_workspace_bytes(...) bytes (two buffer sets of one head group: eight bf16
+ *                    tensors and the LSE block); contents undefined afterwards.
+ *   cuda_stream      the work is ordered after what is already on this stream, and the stream continues only
+ *                    after the last output byte has reached the host; the copies and the kernel themselves run
+ *                    on three streams the library creates once per device.  The call returns when everything is
+ *                    enqueued: host inputs must stay unchanged, and host outputs unread, until the stream has
+ *                    been synchronised.  Calls on one device are serialised on the host by a lock.
+ * Flags, scale and error codes as attn_jvp_fwd; ATTN_JVP_ERR_WORKSPACE if workspace_bytes is too small,
+ * ATTN_JVP_ERR_ALIGN if the workspace is not 256-byte aligned.  Nothing is enqueued unless the arguments check
+ * out; if a CUDA call fails part-way, what was enqueued still completes before the stream continues.
+ */
+size_t attn_jvp_host_workspace_bytes(int B, int H, int Lq, int Lk, int D, int heads_per_stage);
+int attn_jvp_fwd_host(const void* q, const void* k, const void* v,
+                      const void* tq, const void* tk, const void* tv,
+                      void* o, void* to, float* lse,
+                      int B, int H, int Lq, int Lk, int D,
+                      float scale, unsigned flags, int heads_per_stage,
+                      void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /*
  * attn_jvp_fwd_splitkv_static -- the split-KV computation of attn_jvp_fwd_splitkv for callers that are not

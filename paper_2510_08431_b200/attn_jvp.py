@@ -22,7 +22,8 @@ ERR_STATIC_SCRATCH = 13
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 EXPORTS = ("attn_jvp_fwd", "attn_jvp_fwd_stream", "attn_jvp_fwd_mu", "attn_jvp_splitkv_workspace_bytes",
-           "attn_jvp_fwd_splitkv", "attn_jvp_fwd_splitkv_static", "attn_jvp_qknorm_fwd", "attn_jvp_selftest_bounded_wait", "attn_jvp_set_stream", "attn_jvp_device_status", "attn_jvp_strerror",
+           "attn_jvp_fwd_splitkv", "attn_jvp_fwd_splitkv_static", "attn_jvp_host_workspace_bytes",
+           "attn_jvp_fwd_host", "attn_jvp_qknorm_fwd", "attn_jvp_selftest_bounded_wait", "attn_jvp_set_stream", "attn_jvp_device_status", "attn_jvp_strerror",
            "attn_jvp_version")
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libattn_jvp.so")
@@ -64,6 +65,10 @@ def load():
             lib.attn_jvp_fwd_splitkv.restype = ci
             lib.attn_jvp_fwd_splitkv_static.argtypes = [vp] * 10 + [ci] * 5 + [cf, cu, ci, vp]
             lib.attn_jvp_fwd_splitkv_static.restype = ci
+            lib.attn_jvp_host_workspace_bytes.argtypes = [ci] * 6
+            lib.attn_jvp_host_workspace_bytes.restype = ctypes.c_size_t
+            lib.attn_jvp_fwd_host.argtypes = [vp] * 9 + [ci] * 5 + [cf, cu, ci, vp, ctypes.c_size_t, vp]
+            lib.attn_jvp_fwd_host.restype = ci
             lib.attn_jvp_qknorm_fwd.argtypes = [vp] * 5 + [ctypes.c_longlong, ci, cf, vp]
             lib.attn_jvp_qknorm_fwd.restype = ci
             lib.attn_jvp_selftest_bounded_wait.argtypes = [vp]
@@ -232,17 +237,69 @@ def attention_jvp(q, k, v, tq=None, tk=None, tv=None, scale=None, fwd_only=False
     return (o, to, lse, mu) if return_mu else (o, to, lse)
 
 
-def attention_jvp_host(q, k, v, tq=None, tk=None, tv=None, scale=None, fwd_only=False, device="cuda:0"):
-    """Host-to-host convenience: (pinned) CPU bf16 tensors in, CPU tensors out.
+def attn_jvp_host_workspace_bytes(B, H, Lq, Lk, D, heads_per_stage=0) -> int:
+    return int(load().attn_jvp_host_workspace_bytes(B, H, Lq, Lk, D, int(heads_per_stage)))
 
-    Copies the inputs to ``device``, runs :func:`attention_jvp`, copies O, tO, LSE back and
-    synchronises.  Returns (o, to, lse) on the CPU.
+
+def attn_jvp_fwd_host(q, k, v, tq, tk, tv, o, to, lse, B, H, Lq, Lk, D, scale, flags, heads_per_stage, workspace,
+                      workspace_bytes, cuda_stream) -> int:
+    """Raw call on HOST tensors (or integer host addresses); ``workspace`` is device memory.  See include/attn_jvp.h."""
+    return int(load().attn_jvp_fwd_host(_ptr(q), _ptr(k), _ptr(v), _ptr(tq), _ptr(tk), _ptr(tv), _ptr(o), _ptr(to),
+                                        _ptr(lse), B, H, Lq, Lk, D, float(scale), int(flags), int(heads_per_stage),
+                                        _ptr(workspace), int(workspace_bytes), _ptr(cuda_stream)))
+
+
+def attention_jvp_host(q, k, v, tq=None, tk=None, tv=None, scale=None, fwd_only=False, device="cuda:0", out=None,
+                       workspace=None, heads_per_stage=0, synchronize=True):
+    """Host-to-host call: CPU bf16 tensors [B][L][H][D] in (pinned memory lets the copies overlap the kernel),
+    CPU tensors out.
+
+    The library pipelines groups of heads: copy in, kernel, copy out (``attn_jvp_fwd_host``).  ``out`` = (o, to,
+    lse) CPU tensors to fill (allocated pinned if omitted; ``to`` is None with ``fwd_only``); ``workspace`` = a
+    uint8 CUDA tensor of at least ``attn_jvp_host_workspace_bytes(...)`` bytes (allocated if omitted).  With
+    ``synchronize=False`` the call returns once everything is enqueued on the current stream of ``device``.
+    Returns (o, to, lse) on the CPU.
     """
     dev = torch.device(device)
-    up = lambda t: None if t is None else t.to(dev, non_blocking=True)
-    o, to, lse = attention_jvp(up(q), up(k), up(v), up(tq), up(tk), up(tv), scale=scale, fwd_only=fwd_only)
-    res = tuple(None if t is None else t.to("cpu", non_blocking=False) for t in (o, to, lse))
-    st = attn_jvp_device_status()
-    if st != 0:
-        raise AttnJvpError(st, attn_jvp_strerror(st))
-    return res
+    for name, t in (("q", q), ("k", k), ("v", v), ("tq", tq), ("tk", tk), ("tv", tv)):
+        if t is not None:
+            if t.device.type != "cpu" or t.dtype != torch.bfloat16 or not t.is_contiguous() or t.dim() != 4:
+                raise ValueError(f"{name} must be a contiguous CPU bf16 tensor [B][L][H][D]")
+    B, Lq, H, D = q.shape
+    Lk = k.shape[1]
+    if k.shape != (B, Lk, H, D) or v.shape != k.shape:
+        raise ValueError("k and v must be [B][Lk][H][D] with the B, H, D of q")
+    flags = 0
+    if fwd_only:
+        flags |= FWD_ONLY
+        tq = tk = tv = None
+    else:
+        if tq is None or tq.shape != q.shape:
+            raise ValueError("tq (shape of q) is required unless fwd_only")
+        if tk is None and tv is None:
+            flags |= KV_TANGENT_FREE
+        elif tk is None or tv is None or tk.shape != k.shape or tv.shape != k.shape:
+            raise ValueError("tk and tv must both be given (shape of k) or both be None")
+    if scale is None:
+        scale = 1.0 / math.sqrt(D)
+    if out is None:
+        o = torch.empty((B, Lq, H, D), dtype=torch.bfloat16, pin_memory=True)
+        to = None if fwd_only else torch.empty((B, Lq, H, D), dtype=torch.bfloat16, pin_memory=True)
+        lse = torch.empty((B, H, Lq), dtype=torch.float32, pin_memory=True)
+    else:
+        o, to, lse = out
+    need = attn_jvp_host_workspace_bytes(B, H, Lq, Lk, D, heads_per_stage)
+    with torch.cuda.device(dev):
+        if workspace is None:
+            workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+        stream = torch.cuda.current_stream(dev)
+        rc = attn_jvp_fwd_host(q, k, v, tq, tk, tv, o, to, lse, B, H, Lq, Lk, D, scale, flags, heads_per_stage,
+                               workspace, workspace.numel() * workspace.element_size(), stream.cuda_stream)
+        if rc != 0:
+            raise AttnJvpError(rc, attn_jvp_strerror(rc))
+        if synchronize:
+            stream.synchronize()
+            st = attn_jvp_device_status()
+            if st != 0:
+                raise AttnJvpError(st, attn_jvp_strerror(st))
+    return o, to, lse

@@ -6,6 +6,7 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "attn_jvp_kernel.cuh"
 #include "qknorm_jvp.cuh"
@@ -280,6 +281,170 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     return 0;
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Host-buffer pipeline: the heads are processed in groups; while the kernel works on one group, the copy
+// engines bring in the next group's inputs and take out the previous group's outputs.
+// ---------------------------------------------------------------------------------------------
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t in = nullptr, comp = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, in_done[2] = {}, comp_done[2] = {}, out_done[2] = {}, end_in = nullptr,
+                end_comp = nullptr, end_out = nullptr;
+    std::mutex lock;     // one enqueue at a time per device: the events are reused from call to call
+};
+HostPipe g_host_pipe[kMaxDevices];
+
+int host_pipe_setup(HostPipe& hp) {
+    if (hp.ready) return 0;
+    cudaError_t e;
+    cudaStream_t* streams[3] = {&hp.in, &hp.comp, &hp.out};
+    for (cudaStream_t* st : streams) {
+        e = cudaStreamCreateWithFlags(st, cudaStreamNonBlocking);
+        if (e != cudaSuccess) return cuda_fail("cudaStreamCreateWithFlags", e);
+    }
+    cudaEvent_t* events[10] = {&hp.start, &hp.in_done[0], &hp.in_done[1], &hp.comp_done[0], &hp.comp_done[1],
+                               &hp.out_done[0], &hp.out_done[1], &hp.end_in, &hp.end_comp, &hp.end_out};
+    for (cudaEvent_t* ev : events) {
+        e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
+        if (e != cudaSuccess) return cuda_fail("cudaEventCreateWithFlags", e);
+    }
+    hp.ready = true;
+    return 0;
+}
+
+// Heads per pipeline stage: the caller's choice, else about five stages, with copy rows of at least 512 bytes.
+int host_heads_per_stage(int H, int D, int requested) {
+    if (requested > 0) return requested < H ? requested : H;
+    int hg = (H + 4) / 5;
+    const int min_heads = (512 + D * 2 - 1) / (D * 2);
+    if (hg < min_heads) hg = min_heads;
+    return hg < H ? hg : H;
+}
+
+struct HostLayout {
+    size_t nq, nk, nl;     // bytes of one Q-side tensor, one K-side tensor, the LSE block of a head group (padded)
+    size_t set_bytes;      // one buffer set: q, tq, o, to, k, v, tk, tv, lse
+    size_t total;          // two sets
+};
+HostLayout host_layout(int B, int Lq, int Lk, int D, int hg) {
+    auto pad = [](size_t n) { return (n + 255) & ~(size_t)255; };
+    HostLayout L;
+    L.nq = pad((size_t)B * Lq * hg * D * 2);
+    L.nk = pad((size_t)B * Lk * hg * D * 2);
+    L.nl = pad((size_t)B * hg * Lq * 4);
+    L.set_bytes = 4 * L.nq + 4 * L.nk + L.nl;
+    L.total = 2 * L.set_bytes;
+    return L;
+}
+
+int run_host(const void* q, const void* k, const void* v, const void* tq, const void* tk, const void* tv, void* o,
+             void* to, float* lse, int B, int H, int Lq, int Lk, int D, float scale, unsigned flags,
+             int heads_per_stage, void* workspace, size_t workspace_bytes, cudaStream_t stream) {
+    if (flags & ~(ATTN_JVP_KV_TANGENT_FREE | ATTN_JVP_FWD_ONLY)) return ATTN_JVP_ERR_FLAGS;
+    const bool fwd_only = (flags & ATTN_JVP_FWD_ONLY) != 0;
+    const bool jvp_kv = !fwd_only && (flags & ATTN_JVP_KV_TANGENT_FREE) == 0;
+    if (B < 1 || H < 1 || Lq < 1 || Lk < 1 || heads_per_stage < 0) return ATTN_JVP_ERR_SHAPE;
+    if (D != 64 && D != 128) return ATTN_JVP_ERR_UNSUPPORTED_D;
+    if (B > 65535 || H > 65535) return ATTN_JVP_ERR_SHAPE;
+    const long double nq_all = (long double)B * H * Lq * D, nk_all = (long double)B * H * Lk * D;
+    if (nq_all * 2 > 9.0e18L || nk_all * 2 > 9.0e18L) return ATTN_JVP_ERR_SHAPE;
+    if (!q || !k || !v || !o || !lse || !workspace) return ATTN_JVP_ERR_NULL;
+    if (!fwd_only && (!tq || !to)) return ATTN_JVP_ERR_NULL;
+    if (jvp_kv && (!tk || !tv)) return ATTN_JVP_ERR_NULL;
+    if (!std::isfinite(scale)) return ATTN_JVP_ERR_SCALE;
+    if ((uintptr_t)workspace & 255u) return ATTN_JVP_ERR_ALIGN;
+    const int hg = host_heads_per_stage(H, D, heads_per_stage);
+    const HostLayout lay = host_layout(B, Lq, Lk, D, hg);
+    if (workspace_bytes < lay.total) return ATTN_JVP_ERR_WORKSPACE;
+
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail("cudaGetDevice", e);
+    if (dev < 0 || dev >= kMaxDevices) return ATTN_JVP_ERR_ARCH;
+    HostPipe& hp = g_host_pipe[dev];
+    std::lock_guard<std::mutex> guard(hp.lock);
+    if (int rc = host_pipe_setup(hp)) return rc;
+
+    // everything below runs after what the caller has already put on `stream` ...
+    e = cudaEventRecord(hp.start, stream);
+    if (e != cudaSuccess) return cuda_fail("cudaEventRecord", e);
+    cudaStream_t internal[3] = {hp.in, hp.comp, hp.out};
+    for (cudaStream_t st : internal) {
+        e = cudaStreamWaitEvent(st, hp.start, 0);
+        if (e != cudaSuccess) return cuda_fail("cudaStreamWaitEvent", e);
+    }
+
+    const size_t row_host = (size_t)H * D * 2;      // bytes between consecutive (b, l) rows of a host tensor
+    int rc = 0;
+    cudaError_t ce = cudaSuccess;
+    const char* what = nullptr;
+    auto check = [&](cudaError_t err, const char* w) { if (err != cudaSuccess && ce == cudaSuccess) { ce = err; what = w; } };
+    const int n_stages = (H + hg - 1) / hg;
+    for (int g = 0; g < n_stages && rc == 0 && ce == cudaSuccess; ++g) {
+        const int set = g & 1;
+        const int h0 = g * hg;
+        const int hc = (H - h0 < hg) ? H - h0 : hg;
+        char* base = static_cast<char*>(workspace) + (size_t)set * lay.set_bytes;
+        char* d_q = base;
+        char* d_tq = d_q + lay.nq;
+        char* d_o = d_tq + lay.nq;
+        char* d_to = d_o + lay.nq;
+        char* d_k = d_to + lay.nq;
+        char* d_v = d_k + lay.nk;
+        char* d_tk = d_v + lay.nk;
+        char* d_tv = d_tk + lay.nk;
+        float* d_lse = reinterpret_cast<float*>(d_tv + lay.nk);
+        const size_t row_dev = (size_t)hc * D * 2;  // the device copy of a head group is dense: [B][L][hc][D]
+        const size_t head_off = (size_t)h0 * D * 2;
+
+        // inputs of this group: gather the group's heads out of the interleaved host rows
+        if (g >= 2) check(cudaStreamWaitEvent(hp.in, hp.out_done[set], 0), "cudaStreamWaitEvent");
+        auto h2d = [&](char* dst, const void* src, int L) {
+            check(cudaMemcpy2DAsync(dst, row_dev, static_cast<const char*>(src) + head_off, row_host, row_dev,
+                                    (size_t)B * L, cudaMemcpyHostToDevice, hp.in), "cudaMemcpy2DAsync (host to device)");
+        };
+        h2d(d_k, k, Lk);
+        h2d(d_q, q, Lq);
+        if (!fwd_only) h2d(d_tq, tq, Lq);
+        if (jvp_kv) h2d(d_tk, tk, Lk);
+        h2d(d_v, v, Lk);
+        if (jvp_kv) h2d(d_tv, tv, Lk);
+        check(cudaEventRecord(hp.in_done[set], hp.in), "cudaEventRecord");
+        if (ce != cudaSuccess) break;
+
+        // the kernel on the dense group (H = hc)
+        check(cudaStreamWaitEvent(hp.comp, hp.in_done[set], 0), "cudaStreamWaitEvent");
+        if (ce != cudaSuccess) break;
+        rc = run(d_q, d_k, d_v, fwd_only ? nullptr : d_tq, jvp_kv ? d_tk : nullptr, jvp_kv ? d_tv : nullptr, d_o,
+                 fwd_only ? nullptr : d_to, d_lse, nullptr, B, hc, Lq, Lk, D, scale, flags, 1, nullptr, 0, hp.comp);
+        if (rc != 0) break;
+        check(cudaEventRecord(hp.comp_done[set], hp.comp), "cudaEventRecord");
+
+        // outputs of this group: scatter the heads back into the host rows; LSE is [B][H][Lq] on the host
+        check(cudaStreamWaitEvent(hp.out, hp.comp_done[set], 0), "cudaStreamWaitEvent");
+        check(cudaMemcpy2DAsync(static_cast<char*>(o) + head_off, row_host, d_o, row_dev, row_dev, (size_t)B * Lq,
+                                cudaMemcpyDeviceToHost, hp.out), "cudaMemcpy2DAsync (device to host)");
+        if (!fwd_only)
+            check(cudaMemcpy2DAsync(static_cast<char*>(to) + head_off, row_host, d_to, row_dev, row_dev,
+                                    (size_t)B * Lq, cudaMemcpyDeviceToHost, hp.out), "cudaMemcpy2DAsync (device to host)");
+        check(cudaMemcpy2DAsync(lse + (size_t)h0 * Lq, (size_t)H * Lq * 4, d_lse, (size_t)hc * Lq * 4,
+                                (size_t)hc * Lq * 4, (size_t)B, cudaMemcpyDeviceToHost, hp.out),
+              "cudaMemcpy2DAsync (LSE)");
+        check(cudaEventRecord(hp.out_done[set], hp.out), "cudaEventRecord");
+    }
+    // ... and the caller's stream continues after all of it (also when an error cut the loop short)
+    check(cudaEventRecord(hp.end_in, hp.in), "cudaEventRecord");
+    check(cudaEventRecord(hp.end_comp, hp.comp), "cudaEventRecord");
+    check(cudaEventRecord(hp.end_out, hp.out), "cudaEventRecord");
+    check(cudaStreamWaitEvent(stream, hp.end_in, 0), "cudaStreamWaitEvent");
+    check(cudaStreamWaitEvent(stream, hp.end_comp, 0), "cudaStreamWaitEvent");
+    check(cudaStreamWaitEvent(stream, hp.end_out, 0), "cudaStreamWaitEvent");
+    if (rc != 0) return rc;
+    if (ce != cudaSuccess) return cuda_fail(what, ce);
+    return 0;
+}
+
 }  // namespace
 
 extern "C" {
@@ -317,6 +482,18 @@ int attn_jvp_fwd_splitkv(const void* q, const void* k, const void* v, const void
                          unsigned flags, int splits, void* workspace, size_t workspace_bytes, void* cuda_stream) {
     return run(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, Lk, D, scale, flags, splits, workspace, workspace_bytes,
                static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t attn_jvp_host_workspace_bytes(int B, int H, int Lq, int Lk, int D, int heads_per_stage) {
+    if (B < 1 || H < 1 || Lq < 1 || Lk < 1 || (D != 64 && D != 128) || heads_per_stage < 0) return 0;
+    return host_layout(B, Lq, Lk, D, host_heads_per_stage(H, D, heads_per_stage)).total;
+}
+
+int attn_jvp_fwd_host(const void* q, const void* k, const void* v, const void* tq, const void* tk, const void* tv,
+                      void* o, void* to, float* lse, int B, int H, int Lq, int Lk, int D, float scale, unsigned flags,
+                      int heads_per_stage, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+    return run_host(q, k, v, tq, tk, tv, o, to, lse, B, H, Lq, Lk, D, scale, flags, heads_per_stage, workspace,
+                    workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
 }
 
 // Scratch for callers that cannot allocate: lives in the library's device image, so every GPU that loads
@@ -448,7 +625,7 @@ const char* attn_jvp_strerror(int code) {
             return tl_strerror_buf;
         case ATTN_JVP_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait expired; the kernel stopped early";
         case ATTN_JVP_ERR_DEVICE_LAYOUT: return "the kernel's shared-memory layout did not fit; nothing was computed";
-        case ATTN_JVP_ERR_WORKSPACE: return "the split-KV workspace is smaller than attn_jvp_splitkv_workspace_bytes()";
+        case ATTN_JVP_ERR_WORKSPACE: return "the workspace is smaller than the matching *_workspace_bytes() function asks for";
         case ATTN_JVP_ERR_STATIC_SCRATCH:
             snprintf(tl_strerror_buf, sizeof tl_strerror_buf, "built-in scratch too small: %s", tl_cuda_msg);
             return tl_strerror_buf;
