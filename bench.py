@@ -130,8 +130,10 @@ def time_oracle(w, x_host, budget_s: float):
                                    w.B, w.H, w.Lq, w.Lk, w.D, w.scale, rows)
         return len(rows), time.perf_counter() - t0
 
+    # two probes: the first one mostly measures the one-off widening of K, V, tK, tV to fp64
     n0, t_probe = run(64)
-    rate = n0 / max(t_probe, 1e-6)
+    n1, t_probe = run(int(max(64, min(w.Lq, 64 / max(t_probe, 1e-6) * 2.0))))
+    rate = n1 / max(t_probe, 1e-6)
     n = int(max(64, min(n_total, w.Lq, rate * budget_s)))
     n, dt = run(n)
     nominal_per_row = 12 * w.Lk * w.D
