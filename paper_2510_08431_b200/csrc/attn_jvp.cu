@@ -235,7 +235,7 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     // persistent CTAs: one per SM (fewer if there is less work), sharing the work items round-robin
     const long long n_q_tiles = (Lq + attn_jvp::kBlockM - 1) / attn_jvp::kBlockM;
     const long long n_items = n_q_tiles * H * B * eff_splits;
-    if (n_items > 0x7fffffffLL) return ATTN_JVP_ERR_SHAPE;
+    if (n_items > 0x7fffffffLL - 65536) return ATTN_JVP_ERR_SHAPE;   // item + gridDim.x must not overflow an int
     ka.n_q_tiles = (int)n_q_tiles;
     ka.n_items = (int)n_items;
     if (g_sm_count[dev] == 0) {

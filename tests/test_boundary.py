@@ -93,3 +93,42 @@ def test_python_wrapper_validates_tensors(lib):
     q = torch.zeros(1, 8, 2, 64, dtype=torch.bfloat16)
     with pytest.raises(ValueError):
         lib.attention_jvp(q, q, q, q, q, q)  # CPU tensors are refused: there is no CPU path
+
+
+def test_workspace_size_functions_are_plain_host_arithmetic(lib):
+    """Sizes of the two caller-provided workspaces (no GPU involved)."""
+    # split-KV: per chunk fp32 O and tO partials [B][Lq][H][D] and fp32 LSE, mu partials [B][H][Lq] (16-byte padded)
+    B, H, Lq, Lk, D = 1, 8, 512, 32760, 128
+    assert lib.attn_jvp_splitkv_workspace_bytes(B, H, Lq, Lk, D, 1) == 0          # one chunk: the plain kernel
+    four = lib.attn_jvp_splitkv_workspace_bytes(B, H, Lq, Lk, D, 4)
+    assert four == 2 * 4 * B * Lq * H * D * 4 + 2 * 4 * B * H * Lq * 4
+    assert lib.attn_jvp_splitkv_workspace_bytes(B, H, Lq, Lk, 96, 4) == 0
+    # host pipeline: two buffer sets of one head group (4 Q-side + 4 K-side bf16 tensors + LSE, 256-byte padded)
+    pad = lambda n: (n + 255) // 256 * 256
+    for (B, H, Lq, Lk, D, hps, hg) in ((1, 40, 32760, 32760, 128, 0, 8), (1, 40, 32760, 32760, 128, 3, 3),
+                                       (2, 5, 300, 200, 128, 2, 2), (1, 7, 129, 513, 64, 0, 4),
+                                       (1, 3, 50, 60, 64, 0, 3), (1, 2, 50, 60, 128, 9, 2)):
+        want = 2 * (4 * pad(B * Lq * hg * D * 2) + 4 * pad(B * Lk * hg * D * 2) + pad(B * hg * Lq * 4))
+        assert lib.attn_jvp_host_workspace_bytes(B, H, Lq, Lk, D, hps) == want
+    assert lib.attn_jvp_host_workspace_bytes(1, 4, 64, 64, 96, 0) == 0
+    assert lib.attn_jvp_host_workspace_bytes(1, 4, 64, 64, 64, -1) == 0
+
+
+def test_host_entry_point_rejects_bad_arguments_before_any_gpu_work(lib):
+    """attn_jvp_fwd_host validates everything, including the workspace, before it creates a stream or copies."""
+    base = [A, A + STEP, A + 2 * STEP, A + 3 * STEP, A + 4 * STEP, A + 5 * STEP, A + 6 * STEP, A + 7 * STEP,
+            A + 8 * STEP, 1, 4, 128, 128, 128, 0.088, 0, 0]
+    need = lib.attn_jvp_host_workspace_bytes(1, 4, 128, 128, 128, 0)
+    ws = A + 9 * STEP
+
+    def call(args, workspace=ws, nbytes=need):
+        return lib.attn_jvp_fwd_host(*args, workspace, nbytes, None)
+
+    assert call(base, nbytes=need - 1) == 12
+    assert call(base, workspace=ws + 16) == 4
+    assert call(base, workspace=None) == 1
+    for idx, val, code in ((0, None, 1), (3, None, 1), (7, None, 1), (8, None, 1), (15, 0x10, 5), (16, -2, 2),
+                           (9, 0, 2), (13, 80, 3), (14, float("nan"), 6)):
+        bad = list(base)
+        bad[idx] = val
+        assert call(bad) == code, (idx, val)
