@@ -53,7 +53,7 @@ enum Mode : int { kModeJvp = 0, kModeKvTangentFree = 1, kModeFwdOnly = 2 };
 // one CTA stamps clock64() at the hand-over points of its roles for the first kTraceSteps key tiles.
 #ifdef ATTN_JVP_TRACE
 constexpr int kTraceSteps = 96;
-constexpr int kTraceEvents = 24;
+constexpr int kTraceEvents = 32;
 __device__ long long g_trace[kTraceEvents][kTraceSteps];
 #if ATTN_JVP_TRACE >= 2
 #define TRACE(evt, idx) do { if (trace_on && (idx) < kTraceSteps) g_trace[evt][idx] = clock64(); } while (0)
@@ -374,6 +374,11 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // up one slot per output tensor (a slot is exactly one 128 x D bf16 tile).  The split-KV kernel writes its
     // fp32 partial results straight from registers and stages nothing.
     constexpr int kStageSlots = kSplit ? 0 : (kHasTQ ? 2 : 1);
+    // With tK = tV = 0 the tensor pipe has spare time and a key tile takes as long as the chain softmax -> value
+    // MMAs -> score MMAs: there P~ is handed to the MMA warp as soon as it is stored, and the MMAs that read it run
+    // beside the H~ arithmetic (H~ follows through a barrier of its own).  In the full mode the MMA warp never
+    // waits for the softmax warps, and the second hand-over would only add work (measured: 1 % slower).
+    constexpr bool kSplitHandover = kHasTQ && !kHasTKV;
     static_assert(Plan::kSlotBytes == Plan::kQBytes, "an output tile must fill one ring slot");
 
     extern __shared__ uint8_t smem_raw[];
@@ -382,7 +387,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     __shared__ __align__(8) uint64_t bar_slot_full[kSlots];
     __shared__ __align__(8) uint64_t bar_slot_empty[kSlots];
     __shared__ __align__(8) uint64_t bar_s_full[2];
-    __shared__ __align__(8) uint64_t bar_p_full[2];
+    __shared__ __align__(8) uint64_t bar_p_full[2];     // P~ of the tile is in tensor memory
+    __shared__ __align__(8) uint64_t bar_h_full[2];     // H~ of the tile is in tensor memory (some 500 cycles later)
     __shared__ __align__(8) uint64_t bar_pv_done;
     __shared__ __align__(8) uint64_t bar_acc_free;   // the epilogue has read O and T: the next item may overwrite them
     __shared__ __align__(8) uint64_t bar_drain;
@@ -452,6 +458,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         for (int i = 0; i < 2; ++i) {
             mbar_init(smem_u32(&bar_s_full[i]), 1);
             mbar_init(smem_u32(&bar_p_full[i]), kSoftmaxThreads / 32);    // one arrival per softmax warp
+            mbar_init(smem_u32(&bar_h_full[i]), kSoftmaxThreads / 32);
         }
         mbar_init(smem_u32(&bar_pv_done), 1);
         mbar_init(smem_u32(&bar_acc_free), kSoftmaxThreads / 32);
@@ -725,14 +732,18 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 TRACE(2, g);          // MMA: score MMAs of tile g issued
             };
             // value MMAs of tile j of the item (global tile g) out of ring slot `slot`
-            auto issue_values = [&](int j, int g, int slot) {
+            // value MMAs of tile j of the item (global tile g) out of ring slot `slot`, in two parts: those that read
+            // P~ can run while the softmax warps are still forming H~
+            auto issue_values_p = [&](int j, int g) {
                 const uint32_t tm_p = tmem + kScoreCol0 + (g & 1) * kScoreBufStride;
-                const uint32_t tm_h = tm_p + kBlockN;
                 TRACE(3, g);          // MMA: about to issue value MMAs
 #pragma unroll
                 for (int k = 0; k < kBlockN / 16; ++k) {
                     mma_ts(tmem_o, tm_p + k * 8, vd[k], kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
                 }
+            };
+            auto issue_values_h = [&](int j, int g, int slot) {
+                const uint32_t tm_h = tmem + kScoreCol0 + (g & 1) * kScoreBufStride + kBlockN;
                 if (kHasTQ) {
 #pragma unroll
                     for (int k = 0; k < kBlockN / 16; ++k) {
@@ -810,8 +821,22 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         if (nxt_has_k) advance(pos);
                     }
                     tc_fence_after();
+                    if (leader) issue_values_p(j, g0 + j);
+                    __syncwarp();
+                    if (kSplitHandover) {
+                        // H~ follows P~ by a few hundred cycles: normally it is there by now
+                        const uint32_t hbar = smem_u32(&bar_h_full[(g0 + j) & 1]);
+                        const uint32_t hpar = ((g0 + j) >> 1) & 1;
+                        if (!__all_sync(0xffffffffu, mbar_test_wait(hbar, hpar))) {
+                            if (leader) TRACE(24, g0 + j);   // MMA: has to block for H~ of tile g
+                            ok = mbar_wait_warp(hbar, hpar, abort_state);
+                            if (leader) TRACE(25, g0 + j);   // MMA: H~ of tile g seen
+                            if (!ok) break;
+                        }
+                        tc_fence_after();
+                    }
                     if (leader) {
-                        issue_values(j, g0 + j, pos_v.slot);
+                        issue_values_h(j, g0 + j, pos_v.slot);
                         if (has_k) issue_scores_a(g0 + j + 2);
                     }
                     __syncwarp();
@@ -966,6 +991,13 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     for (int c = 0; c < kBlockN / 2; ++c) pk[c] = pack_bf16(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1]));
                     TMEM_ST32(tm_s, pk, 0);
                 }
+                if (kSplitHandover) {
+                    // P~ is handed over at once: the MMAs that read it run beside the H~ arithmetic below
+                    tc_wait_st();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bar_p_full[bsel]));
+                }
                 if (kHasTQ) {
                     // tO does not change when a per-row constant is subtracted from tS (softmax is shift
                     // invariant: the constant leaves H~ V - (r/l) O unchanged).  Centring tS on its P-weighted
@@ -1006,7 +1038,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bar_p_full[bsel]));
+                if (lane == 0) mbar_arrive(smem_u32(kSplitHandover ? &bar_h_full[bsel] : &bar_p_full[bsel]));
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
                 if (trace_me && g < kTraceSteps) g_trace[13 + ((warp - kFirstSoftmaxWarp) & 3)][g] = clock64();    // softmax warp: arrived
 #endif
