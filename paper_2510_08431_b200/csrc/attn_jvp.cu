@@ -140,7 +140,7 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     const int mode = fwd_only ? attn_jvp::kModeFwdOnly : (kv_free ? attn_jvp::kModeKvTangentFree : attn_jvp::kModeJvp);
     if (B < 1 || H < 1 || Lq < 1 || Lk < 1) return ATTN_JVP_ERR_SHAPE;
     if (D != 64 && D != 128) return ATTN_JVP_ERR_UNSUPPORTED_D;
-    if (B > 65535 || H > 65535) return ATTN_JVP_ERR_SHAPE;   // grid y / z limits
+    if (B > 65535 || H > 65535) return ATTN_JVP_ERR_SHAPE;   // documented limits of the interface
     const long double nq = (long double)B * H * Lq * D, nk = (long double)B * H * Lk * D;
     if (nq * 2 > 9.0e18L || nk * 2 > 9.0e18L) return ATTN_JVP_ERR_SHAPE;
     if (!q || !k || !v || !o || !lse) return ATTN_JVP_ERR_NULL;

@@ -78,7 +78,8 @@ struct KernelArgs {
     float scale_log2;   // s * log2(e)
     // optional side output: mu = rowsum(P . tS) = d(LSE) along the tangent, fp32 [B][H][Lq] (may be null)
     float* mu;
-    // split-KV mode: the keys are cut into `splits` chunks of `tiles_per_split` tiles; blockIdx.z = b * splits + s;
+    // split-KV mode: the keys are cut into `splits` chunks of `tiles_per_split` tiles; a work item is then one
+    // (query tile, head, batch, chunk);
     // chunk s writes normalised partial results (fp32) instead of the final outputs
     int splits;
     int tiles_per_split;
