@@ -50,7 +50,7 @@ extern "C" {
 /* error codes */
 #define ATTN_JVP_OK                  0
 #define ATTN_JVP_ERR_NULL            1  /* a required pointer is NULL */
-#define ATTN_JVP_ERR_SHAPE           2  /* B, H, Lq or Lk < 1, or sizes overflow */
+#define ATTN_JVP_ERR_SHAPE           2  /* B, H, Lq or Lk < 1; B or H > 65535; sizes overflow; bad splits / heads_per_stage */
 #define ATTN_JVP_ERR_UNSUPPORTED_D   3  /* D is not 64 or 128 */
 #define ATTN_JVP_ERR_ALIGN           4  /* a tensor pointer is not 16-byte aligned */
 #define ATTN_JVP_ERR_FLAGS           5  /* unknown flag bits */
