@@ -138,7 +138,8 @@ int attn_jvp_fwd_splitkv(const void* q, const void* k, const void* v,
  *   heads_per_stage  heads per pipeline stage; 0 = library default (about five stages, copy rows >= 512 bytes).
  *   workspace        DEVICE scratch owned by the caller, 256-byte aligned, at least
  *                    attn_jvp_host_workspace_bytes(...) bytes (two buffer sets of one head group: eight bf16
- *                    tensors and the LSE block); contents undefined afterwards.
+ *                    tensors and the LSE block); contents undefined afterwards.  Two calls that share a
+ *                    workspace must be ordered on the GPU (same stream, or an event between their streams).
  *   cuda_stream      the work is ordered after what is already on this stream, and the stream continues only
  *                    after the last output byte has reached the host; the copies and the kernel themselves run
  *                    on three streams the library creates once per device.  The call returns when everything is
