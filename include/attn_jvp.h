@@ -117,6 +117,11 @@ int attn_jvp_fwd_mu(const void* q, const void* k, const void* v,
  * Returns ATTN_JVP_ERR_WORKSPACE if workspace_bytes is too small.
  */
 size_t attn_jvp_splitkv_workspace_bytes(int B, int H, int Lq, int Lk, int D, int splits);
+/* A number of chunks for attn_jvp_fwd_splitkv that fills the current device: 1 when the query tiles alone keep
+ * at least ~60 % of the SMs busy, else the largest count for which (query tiles x heads x batch x chunks) still
+ * fits one wave of CTAs, with at least four 64-key tiles per chunk.  (A heuristic of this library, measured on
+ * B200; the paper has no counterpart.)  Returns 1 for invalid shapes or when no CUDA device is current. */
+int attn_jvp_suggest_splits(int B, int H, int Lq, int Lk, int D);
 int attn_jvp_fwd_splitkv(const void* q, const void* k, const void* v,
                          const void* tq, const void* tk, const void* tv,
                          void* o, void* to, float* lse, float* mu,

@@ -22,7 +22,7 @@ ERR_STATIC_SCRATCH = 13
 STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 EXPORTS = ("attn_jvp_fwd", "attn_jvp_fwd_stream", "attn_jvp_fwd_mu", "attn_jvp_splitkv_workspace_bytes",
-           "attn_jvp_fwd_splitkv", "attn_jvp_fwd_splitkv_static", "attn_jvp_host_workspace_bytes",
+           "attn_jvp_suggest_splits", "attn_jvp_fwd_splitkv", "attn_jvp_fwd_splitkv_static", "attn_jvp_host_workspace_bytes",
            "attn_jvp_fwd_host", "attn_jvp_qknorm_fwd", "attn_jvp_selftest_bounded_wait", "attn_jvp_set_stream", "attn_jvp_device_status", "attn_jvp_strerror",
            "attn_jvp_version")
 
@@ -61,6 +61,8 @@ def load():
             lib.attn_jvp_fwd_mu.restype = ci
             lib.attn_jvp_splitkv_workspace_bytes.argtypes = [ci] * 6
             lib.attn_jvp_splitkv_workspace_bytes.restype = ctypes.c_size_t
+            lib.attn_jvp_suggest_splits.argtypes = [ci] * 5
+            lib.attn_jvp_suggest_splits.restype = ci
             lib.attn_jvp_fwd_splitkv.argtypes = [vp] * 10 + [ci] * 5 + [cf, cu, ci, vp, ctypes.c_size_t, vp]
             lib.attn_jvp_fwd_splitkv.restype = ci
             lib.attn_jvp_fwd_splitkv_static.argtypes = [vp] * 10 + [ci] * 5 + [cf, cu, ci, vp]
@@ -136,6 +138,10 @@ def attn_jvp_splitkv_workspace_bytes(B, H, Lq, Lk, D, splits) -> int:
     return int(load().attn_jvp_splitkv_workspace_bytes(B, H, Lq, Lk, D, splits))
 
 
+def attn_jvp_suggest_splits(B, H, Lq, Lk, D) -> int:
+    return int(load().attn_jvp_suggest_splits(B, H, Lq, Lk, D))
+
+
 def attn_jvp_fwd_splitkv(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, Lk, D, scale, flags, splits, workspace,
                          workspace_bytes, cuda_stream) -> int:
     return int(load().attn_jvp_fwd_splitkv(_ptr(q), _ptr(k), _ptr(v), _ptr(tq), _ptr(tk), _ptr(tv), _ptr(o),
@@ -193,7 +199,8 @@ def attention_jvp(q, k, v, tq=None, tk=None, tv=None, scale=None, fwd_only=False
     context); ``fwd_only`` runs the plain forward (returns tO = None).  ``out`` may supply
     preallocated (o, to, lse).  ``return_mu`` adds mu = rowsum(P . tS) (the tangent of LSE) as a fourth
     result.  ``splits`` > 1 cuts the keys into chunks processed by independent CTAs and merged by a
-    second kernel (for few queries and many keys); ``workspace`` may supply its scratch (a CUDA uint8
+    second kernel (for few queries and many keys), ``splits=0`` lets the library choose
+    (``attn_jvp_suggest_splits``); ``workspace`` may supply its scratch (a CUDA uint8
     tensor of at least attn_jvp_splitkv_workspace_bytes), else it is allocated here with torch.
     Returns (o, to, lse) or (o, to, lse, mu).
     """
@@ -221,6 +228,8 @@ def attention_jvp(q, k, v, tq=None, tk=None, tv=None, scale=None, fwd_only=False
     mu = torch.empty((B, H, Lq), dtype=torch.float32, device=q.device) if return_mu else None
     with torch.cuda.device(q.device):
         stream = torch.cuda.current_stream().cuda_stream
+        if splits == 0:
+            splits = attn_jvp_suggest_splits(B, H, Lq, Lk, D)
         if splits > 1:
             need = attn_jvp_splitkv_workspace_bytes(B, H, Lq, Lk, D, splits)
             if workspace is None and need > 0:

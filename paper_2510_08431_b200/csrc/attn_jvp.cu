@@ -477,6 +477,25 @@ size_t attn_jvp_splitkv_workspace_bytes(int B, int H, int Lq, int Lk, int D, int
     return split_layout(B, H, Lq, D, eff).total;
 }
 
+int attn_jvp_suggest_splits(int B, int H, int Lq, int Lk, int D) {
+    if (B < 1 || H < 1 || Lq < 1 || Lk < 1 || (D != 64 && D != 128)) return 1;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+        (void)cudaGetLastError();
+        return 1;
+    }
+    // Work items without a split; with at least ~60 % of the SMs busy a split only adds the merge.
+    const long long items = (long long)((Lq + attn_jvp::kBlockM - 1) / attn_jvp::kBlockM) * H * B;
+    if (items * 5 >= (long long)sms * 3) return 1;
+    // Otherwise: the largest number of chunks that still fits one wave of CTAs, with at least four key tiles each.
+    const int n_tiles = (Lk + attn_jvp::kBlockN - 1) / attn_jvp::kBlockN;
+    long long splits = sms / items;
+    if (splits > n_tiles / 4) splits = n_tiles / 4;
+    if (splits > 1024) splits = 1024;
+    return splits < 1 ? 1 : (int)splits;
+}
+
 int attn_jvp_fwd_splitkv(const void* q, const void* k, const void* v, const void* tq, const void* tk, const void* tv,
                          void* o, void* to, float* lse, float* mu, int B, int H, int Lq, int Lk, int D, float scale,
                          unsigned flags, int splits, void* workspace, size_t workspace_bytes, void* cuda_stream) {

@@ -132,3 +132,11 @@ def test_host_entry_point_rejects_bad_arguments_before_any_gpu_work(lib):
         bad = list(base)
         bad[idx] = val
         assert call(bad) == code, (idx, val)
+
+
+def test_suggest_splits_is_one_without_a_device_or_for_bad_shapes(lib):
+    import torch
+    assert lib.attn_jvp_suggest_splits(1, 8, 512, 32760, 96) == 1
+    assert lib.attn_jvp_suggest_splits(0, 8, 512, 32760, 128) == 1
+    if not torch.cuda.is_available():
+        assert lib.attn_jvp_suggest_splits(1, 8, 512, 32760, 128) == 1

@@ -100,3 +100,23 @@ def test_layer_front_end_matches_direct_calls(aj):
     assert torch.equal(o_plain, ro) and torch.equal(oc, rco) and torch.equal(toc, rcto)
     with pytest.raises(ValueError):
         layer((g["q"], g["tq"]), (g["k"], g["tk"]), g["v"], withT=True)
+
+
+def test_suggested_splits_fill_one_wave_and_give_the_same_result(aj, oracle):
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    # plenty of query tiles: no split
+    assert aj.attn_jvp_suggest_splits(1, 40, 32760, 32760, 128) == 1
+    assert aj.attn_jvp_suggest_splits(2, 8, 2048, 4096, 128) == 1
+    # few query tiles: the largest chunk count that fits one wave, at least four key tiles per chunk
+    B, H, Lq, Lk, D = 1, 8, 512, 8192, 128
+    items = (Lq + 127) // 128 * H * B
+    want = max(1, min(sms // items, (Lk + 63) // 64 // 4))
+    assert aj.attn_jvp_suggest_splits(B, H, Lq, Lk, D) == want
+    assert aj.attn_jvp_suggest_splits(1, 1, 64, 1024, 64) == 4          # 16 key tiles: four per chunk
+    x = synth.make_inputs(B, H, Lq, Lk, D, 1.0, 0.5, seed=77)
+    g = U.to_gpu(x)
+    o, to, lse = aj.attention_jvp(g["q"], g["k"], g["v"], g["tq"], g["tk"], g["tv"], splits=0)
+    torch.cuda.synchronize()
+    assert aj.attn_jvp_device_status() == 0
+    rows = synth.sample_rows(B, H, Lq, n_random_per_head=8, seed=3)
+    U.check_all(oracle, aj, x, B, H, Lq, Lk, D, D ** -0.5, rows, o, to, lse)
