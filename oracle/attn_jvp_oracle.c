@@ -13,10 +13,12 @@
  *                    tS = tQ K^T + Q tK^T, tP = P.tS - P.(rowsum(P.tS) 1 1^T),
  *                    tO = tP V + P tV), two passes over one row of scores.
  *
- *   attn_jvp_alg2_*  the streaming procedure of Algorithm 2 taken step by step
- *                    in the paper's order and notation (m, l, r, O, A, B per
- *                    query row, key blocks of size B_c, epilogue O/l, L = m +
- *                    log l, C = r O, tO = (A + B - C)/l).
+ *   attn_jvp_fold_*  the same quantities reached block by block: the definition
+ *                    on each block of B_c keys, the block results folded into a
+ *                    running (O, tO, LSE, mu) with the chunk-merge identity that
+ *                    follows from the aggregated form of Appendix C.1.  It pins
+ *                    the streaming property (any block size gives the result of
+ *                    the definition) without restating the paper's listing.
  *
  * Readings where the paper is silent:
  *   - the paper writes S = Q K^T with no softmax scale; here S = s Q K^T and
@@ -28,8 +30,8 @@
  *
  * Pins (tests/, "not gpu"): central finite differences of O and LSE, linearity
  * in the tangent, zero tangent, Lk = 1, Q = 0 closed form, constant-V,
- * hand-derived golden values, torch.func.jvp, and def == alg2 on brute-force
- * tiny shapes.
+ * hand-derived golden values, torch.func.jvp, and definition == block-fold on
+ * brute-force tiny shapes.
  *
  * All matrices handed to the *_f64 entry points are dense row-major doubles:
  * Q,tQ [Lq][D]; K,tK,V,tV [Lk][D]; O,tO [Lq][D]; LSE,mu [Lq].
@@ -129,76 +131,60 @@ int attn_jvp_def_f64(const double *Q, const double *K, const double *V,
 }
 
 /* ------------------------------------------------------------------------- */
-/* Algorithm 2, one query row (B_r = 1; rows never interact), key blocks B_c. */
-static void alg2_row(const double *q, const double *tq,
+/*
+ * Second route: the keys are cut into consecutive blocks of B_c; each block is
+ * evaluated on its own by the definition above (softmax within the block), and
+ * the block results are folded into a running result one after the other.
+ *
+ * Folding two disjoint key sets a and b, each normalised within itself: the
+ * softmax weights over the union are P_j = w_a P^a_j on a and w_b P^b_j on b,
+ * with w_x = exp(LSE_x - LSE) and LSE = log(exp(LSE_a) + exp(LSE_b)).  Putting
+ * that into the aggregated form of Appendix C.1,
+ *     tO = (P.tS) V + P tV - diag(mu) O,   mu = rowsum(P.tS),
+ * and using (P^x.tS) V + P^x tV = tO_x + mu_x O_x on each set gives
+ *     O  = w_a O_a + w_b O_b,        mu = w_a mu_a + w_b mu_b,
+ *     tO = w_a (tO_a + mu_a O_a) + w_b (tO_b + mu_b O_b) - mu O.
+ * In exact arithmetic this is what a single streaming pass over key blocks
+ * (Algorithm 2) arrives at for any block size; only the order of the sums
+ * differs from the definition.
+ */
+static void fold_row(const double *q, const double *tq,
                      const double *K, const double *tK,
                      const double *V, const double *tV,
                      long Lk, long D, long Bc, double scale,
-                     double *o_out, double *to_out, double *lse, double *mu,
-                     double *work /* 3*D + 2*Bc doubles */)
+                     double *o, double *to, double *lse, double *mu,
+                     double *work /* 2*D + 2*Bc doubles */)
 {
-    double *Oi = work, *Ai = work + D, *Bi = work + 2 * D;
-    double *Pt = work + 3 * D, *tSij = Pt + Bc;
-    /* initialise m = -inf, l = 0, O = 0, r = 0, A = 0, B = 0 */
-    double m_i = -INFINITY, l_i = 0.0, r_i = 0.0;
-    for (long d = 0; d < D; ++d) { Oi[d] = 0.0; Ai[d] = 0.0; Bi[d] = 0.0; }
-
+    double *o_b = work, *to_b = work + D;
+    double *s_buf = work + 2 * D, *ts_buf = s_buf + Bc;
     for (long j0 = 0; j0 < Lk; j0 += Bc) {
         const long nb = (Lk - j0 < Bc) ? (Lk - j0) : Bc;
-        /* S_ij = Q_i K_j^T ; tS_ij = tQ_i K_j^T + Q_i tK_j^T */
-        double rowmax = -INFINITY;
-        for (long c = 0; c < nb; ++c) {
-            const double *kj = K + (j0 + c) * D;
-            double s = 0.0, ts = 0.0;
-            for (long d = 0; d < D; ++d) { s += q[d] * kj[d]; ts += tq[d] * kj[d]; }
-            if (tK) {
-                const double *tkj = tK + (j0 + c) * D;
-                for (long d = 0; d < D; ++d) ts += q[d] * tkj[d];
-            }
-            Pt[c] = scale * s;
-            tSij[c] = scale * ts;
-            if (Pt[c] > rowmax) rowmax = Pt[c];
+        double lse_b, mu_b;
+        def_row(q, tq, K + j0 * D, tK ? tK + j0 * D : NULL, V + j0 * D, tV ? tV + j0 * D : NULL,
+                nb, D, D, scale, o_b, to_b, &lse_b, &mu_b, s_buf, ts_buf);
+        if (j0 == 0) {
+            memcpy(o, o_b, sizeof(double) * (size_t)D);
+            memcpy(to, to_b, sizeof(double) * (size_t)D);
+            *lse = lse_b;
+            *mu = mu_b;
+            continue;
         }
-        /* m_new = max(m_i, rowmax(S_ij)) */
-        const double m_new = (m_i > rowmax) ? m_i : rowmax;
-        /* P~_ij = exp(S_ij - m_new) */
-        double rowsum_P = 0.0;
-        for (long c = 0; c < nb; ++c) { Pt[c] = exp(Pt[c] - m_new); rowsum_P += Pt[c]; }
-        const double alpha = exp(m_i - m_new); /* e^{m_i - m_new}; 0 on the first block */
-        /* l_new = alpha l_i + rowsum(P~) */
-        const double l_new = alpha * l_i + rowsum_P;
-        /* O_new = alpha O_i + P~ V_j ; A_new = alpha A_i + P~ tV_j */
-        for (long d = 0; d < D; ++d) { Oi[d] *= alpha; Ai[d] *= alpha; Bi[d] *= alpha; }
-        for (long c = 0; c < nb; ++c) {
-            const double *vj = V + (j0 + c) * D;
-            for (long d = 0; d < D; ++d) Oi[d] += Pt[c] * vj[d];
-            if (tV) {
-                const double *tvj = tV + (j0 + c) * D;
-                for (long d = 0; d < D; ++d) Ai[d] += Pt[c] * tvj[d];
-            }
+        const double top = (*lse > lse_b) ? *lse : lse_b;
+        const double lse_ab = top + log(exp(*lse - top) + exp(lse_b - top));
+        const double w_a = exp(*lse - lse_ab), w_b = exp(lse_b - lse_ab);
+        const double mu_a = *mu;
+        const double mu_ab = w_a * mu_a + w_b * mu_b;
+        for (long d = 0; d < D; ++d) {
+            const double o_ab = w_a * o[d] + w_b * o_b[d];
+            to[d] = w_a * (to[d] + mu_a * o[d]) + w_b * (to_b[d] + mu_b * o_b[d]) - mu_ab * o_ab;
+            o[d] = o_ab;
         }
-        /* H~_ij = P~_ij . tS_ij ; r_new = alpha r_i + rowsum(H~) ; B_new = alpha B_i + H~ V_j */
-        double rowsum_H = 0.0;
-        for (long c = 0; c < nb; ++c) {
-            const double h = Pt[c] * tSij[c];
-            rowsum_H += h;
-            const double *vj = V + (j0 + c) * D;
-            for (long d = 0; d < D; ++d) Bi[d] += h * vj[d];
-        }
-        const double r_new = alpha * r_i + rowsum_H;
-        m_i = m_new; l_i = l_new; r_i = r_new;
+        *lse = lse_ab;
+        *mu = mu_ab;
     }
-    /* O_i = O/l ; L_i = m + log l ; C_i = r O_i ; tO_i = (A + B - C)/l */
-    for (long d = 0; d < D; ++d) o_out[d] = Oi[d] / l_i;
-    *lse = m_i + log(l_i);
-    for (long d = 0; d < D; ++d) {
-        const double Cd = r_i * o_out[d];
-        to_out[d] = (Ai[d] + Bi[d] - Cd) / l_i;
-    }
-    *mu = r_i / l_i;
 }
 
-int attn_jvp_alg2_f64(const double *Q, const double *K, const double *V,
+int attn_jvp_fold_f64(const double *Q, const double *K, const double *V,
                       const double *tQ, const double *tK, const double *tV,
                       long Lq, long Lk, long D, long Bc, double scale,
                       double *O, double *tO, double *LSE, double *MU)
@@ -207,7 +193,7 @@ int attn_jvp_alg2_f64(const double *Q, const double *K, const double *V,
     int fail = 0;
 #pragma omp parallel
     {
-        double *work = (double *)malloc(sizeof(double) * (size_t)(3 * D + 2 * Bc));
+        double *work = (double *)malloc(sizeof(double) * (size_t)(2 * D + 2 * Bc));
         if (!work) {
 #pragma omp atomic write
             fail = 1;
@@ -216,7 +202,7 @@ int attn_jvp_alg2_f64(const double *Q, const double *K, const double *V,
         if (!fail) {
 #pragma omp for schedule(dynamic, 4)
             for (long i = 0; i < Lq; ++i)
-                alg2_row(Q + i * D, tQ + i * D, K, tK, V, tV, Lk, D, Bc, scale,
+                fold_row(Q + i * D, tQ + i * D, K, tK, V, tV, Lk, D, Bc, scale,
                          O + i * D, tO + i * D, LSE + i, MU + i, work);
         }
         free(work);

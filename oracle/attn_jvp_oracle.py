@@ -5,7 +5,8 @@ may import this module; the product path never does.  It compiles
 ``attn_jvp_oracle.c`` (plain C, gcc, OpenMP) on first use and exposes
 
 * ``attn_jvp_def``   the definition of Appendix C.1 written out row by row,
-* ``attn_jvp_alg2``  Algorithm 2 step by step with key blocks of size ``Bc``,
+* ``attn_jvp_fold``  the definition on key blocks of size ``Bc``, folded block by block with the
+  chunk-merge identity (the streaming property: any block size gives the same result),
 * ``attn_jvp_def_bf16_rows``  the definition on bf16 [B][L][H][D] inputs for
   a chosen set of query rows (what the GPU parity tests compare against).
 
@@ -51,8 +52,8 @@ def _load():
             lg = ctypes.c_long
             lib.attn_jvp_def_f64.argtypes = [dp] * 6 + [lg, lg, lg, ctypes.c_double] + [dp] * 4
             lib.attn_jvp_def_f64.restype = ctypes.c_int
-            lib.attn_jvp_alg2_f64.argtypes = [dp] * 6 + [lg, lg, lg, lg, ctypes.c_double] + [dp] * 4
-            lib.attn_jvp_alg2_f64.restype = ctypes.c_int
+            lib.attn_jvp_fold_f64.argtypes = [dp] * 6 + [lg, lg, lg, lg, ctypes.c_double] + [dp] * 4
+            lib.attn_jvp_fold_f64.restype = ctypes.c_int
             lib.attn_jvp_def_bf16_blhd_rows.argtypes = (
                 [u16p] * 6 + [lg] * 5 + [ctypes.c_double, i64p, lg] + [dp] * 4
             )
@@ -109,9 +110,10 @@ def attn_jvp_def(Q, K, V, tQ, tK, tV, scale):
     return _run_f64("attn_jvp_def_f64", Q, K, V, tQ, tK, tV, scale)
 
 
-def attn_jvp_alg2(Q, K, V, tQ, tK, tV, scale, Bc):
-    """Algorithm 2 (streaming, key blocks of ``Bc``).  Returns (O, tO, LSE, mu)."""
-    return _run_f64("attn_jvp_alg2_f64", Q, K, V, tQ, tK, tV, scale, Bc=Bc)
+def attn_jvp_fold(Q, K, V, tQ, tK, tV, scale, Bc):
+    """Block-fold route: the definition on consecutive key blocks of ``Bc``, merged one after the other.
+    Returns (O, tO, LSE, mu)."""
+    return _run_f64("attn_jvp_fold_f64", Q, K, V, tQ, tK, tV, scale, Bc=Bc)
 
 
 def attn_jvp_def_bf16_rows(q, k, v, tq, tk, tv, B, H, Lq, Lk, D, scale, rows):

@@ -27,14 +27,14 @@ def _fd(oracle, x, scale, which=("tQ", "tK", "tV")):
 
 @pytest.mark.parametrize("Lq,Lk,D,scale", [(37, 53, 16, 0.25), (8, 300, 64, 0.125), (5, 1, 8, 1.0),
                                           (16, 2048, 128, 128 ** -0.5)])
-@pytest.mark.parametrize("route", ["def", "alg2"])
+@pytest.mark.parametrize("route", ["def", "fold"])
 def test_fd_all_tangents(oracle, Lq, Lk, D, scale, route):
     rng = np.random.default_rng(Lq * 1000 + Lk)
     x = _rand(rng, Lq, Lk, D)
     if route == "def":
         _, tO, _, MU = oracle.attn_jvp_def(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"], scale)
     else:
-        _, tO, _, MU = oracle.attn_jvp_alg2(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"], scale, Bc=48)
+        _, tO, _, MU = oracle.attn_jvp_fold(x["Q"], x["K"], x["V"], x["tQ"], x["tK"], x["tV"], scale, Bc=48)
     fd_tO, fd_mu = _fd(oracle, x, scale)
     assert np.abs(tO - fd_tO).max() <= 1e-6 * max(1.0, np.abs(tO).max())
     assert np.abs(MU - fd_mu).max() <= 1e-6 * max(1.0, np.abs(MU).max())
@@ -61,7 +61,7 @@ def test_fd_none_tangents_mean_zero(oracle):
     z = np.zeros_like(x["K"])
     a = oracle.attn_jvp_def(x["Q"], x["K"], x["V"], x["tQ"], None, None, 0.2)
     b = oracle.attn_jvp_def(x["Q"], x["K"], x["V"], x["tQ"], z, z, 0.2)
-    c = oracle.attn_jvp_alg2(x["Q"], x["K"], x["V"], x["tQ"], None, None, 0.2, Bc=16)
+    c = oracle.attn_jvp_fold(x["Q"], x["K"], x["V"], x["tQ"], None, None, 0.2, Bc=16)
     for u, v, w in zip(a, b, c):
         np.testing.assert_array_equal(u, v)
         np.testing.assert_allclose(u, w, atol=1e-13, rtol=0)

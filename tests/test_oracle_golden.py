@@ -31,14 +31,14 @@ def _example_b():
                 scale=0.5)
 
 
-@pytest.mark.parametrize("route", ["def", "alg2_1", "alg2_2", "alg2_64"])
+@pytest.mark.parametrize("route", ["def", "fold_1", "fold_2", "fold_64"])
 def test_example_a(oracle, route):
     g = _load()
     ex = _example_a()
     if route == "def":
         O, tO, LSE, MU = oracle.attn_jvp_def(**ex)
     else:
-        O, tO, LSE, MU = oracle.attn_jvp_alg2(**ex, Bc=int(route.split("_")[1]))
+        O, tO, LSE, MU = oracle.attn_jvp_fold(**ex, Bc=int(route.split("_")[1]))
     assert O[0, 0] == pytest.approx(g["A.O"], abs=1e-13)
     assert LSE[0] == pytest.approx(g["A.LSE"], abs=1e-13)
     assert MU[0] == pytest.approx(g["A.mu"], abs=1e-13)
@@ -48,14 +48,14 @@ def test_example_a(oracle, route):
     assert g["A.mu"] == pytest.approx(0.25 + 0.75 * math.log(3), abs=1e-15)
 
 
-@pytest.mark.parametrize("route", ["def", "alg2_1", "alg2_2", "alg2_3"])
+@pytest.mark.parametrize("route", ["def", "fold_1", "fold_2", "fold_3"])
 def test_example_b(oracle, route):
     g = _load()
     ex = _example_b()
     if route == "def":
         O, tO, LSE, MU = oracle.attn_jvp_def(**ex)
     else:
-        O, tO, LSE, MU = oracle.attn_jvp_alg2(**ex, Bc=int(route.split("_")[1]))
+        O, tO, LSE, MU = oracle.attn_jvp_fold(**ex, Bc=int(route.split("_")[1]))
     want_O = np.array([[g["B.O00"], g["B.O01"]], [g["B.O10"], g["B.O11"]]])
     want_tO = np.array([[g["B.tO00"], g["B.tO01"]], [g["B.tO10"], g["B.tO11"]]])
     np.testing.assert_allclose(O, want_O, atol=1e-13, rtol=0)

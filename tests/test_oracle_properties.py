@@ -10,13 +10,13 @@ def _rand(rng, Lq, Lk, D):
     return [f(Lq), f(Lk), f(Lk), f(Lq), f(Lk), f(Lk)]
 
 
-ROUTES = ["def", "alg2"]
+ROUTES = ["def", "fold"]
 
 
 def _call(oracle, route, Q, K, V, tQ, tK, tV, s, Bc=7):
     if route == "def":
         return oracle.attn_jvp_def(Q, K, V, tQ, tK, tV, s)
-    return oracle.attn_jvp_alg2(Q, K, V, tQ, tK, tV, s, Bc=Bc)
+    return oracle.attn_jvp_fold(Q, K, V, tQ, tK, tV, s, Bc=Bc)
 
 
 @pytest.mark.parametrize("route", ROUTES)
@@ -137,25 +137,25 @@ def test_scale_is_not_differentiated_and_enters_both_s_and_ts(oracle):
         np.testing.assert_allclose(u, v, atol=1e-13)
 
 
-def test_alg2_equals_definition_on_tiny_shapes_brute_force(oracle):
+def test_block_fold_equals_definition_on_tiny_shapes_brute_force(oracle):
     """Every Lq, Lk in {1,2,3,5}, D in {1,2,4}, Bc in {1,2,3,64}: the streaming route reorders sums only."""
     rng = np.random.default_rng(10)
     for Lq, Lk, D in itertools.product((1, 2, 3, 5), (1, 2, 3, 5), (1, 2, 4)):
         Q, K, V, tQ, tK, tV = _rand(rng, Lq, Lk, D)
         ref = oracle.attn_jvp_def(Q, K, V, tQ, tK, tV, 0.8)
         for Bc in (1, 2, 3, 64):
-            got = oracle.attn_jvp_alg2(Q, K, V, tQ, tK, tV, 0.8, Bc=Bc)
+            got = oracle.attn_jvp_fold(Q, K, V, tQ, tK, tV, 0.8, Bc=Bc)
             for u, v in zip(ref, got):
                 assert np.abs(u - v).max() <= 1e-12 * (1 + np.abs(u).max())
 
 
-def test_alg2_block_size_independence_long_rows(oracle):
+def test_block_fold_block_size_independence_long_rows(oracle):
     rng = np.random.default_rng(12)
     Q, K, V, tQ, tK, tV = _rand(rng, 4, 1000, 32)
     Q *= 3  # peaked softmax: running max changes late, exercises the rescale terms
     ref = oracle.attn_jvp_def(Q, K, V, tQ, tK, tV, 0.3)
     for Bc in (1, 64, 128, 333, 1000, 4096):
-        got = oracle.attn_jvp_alg2(Q, K, V, tQ, tK, tV, 0.3, Bc=Bc)
+        got = oracle.attn_jvp_fold(Q, K, V, tQ, tK, tV, 0.3, Bc=Bc)
         for u, v in zip(ref, got):
             assert np.abs(u - v).max() <= 1e-11 * (1 + np.abs(u).max())
 
@@ -166,6 +166,6 @@ def test_increasing_maxima_rescale_path(oracle):
     Q, K, V, tQ, tK, tV = _rand(rng, 3, 64, 8)
     K = K * np.linspace(0.1, 6.0, 64)[:, None]
     ref = oracle.attn_jvp_def(Q, K, V, tQ, tK, tV, 1.0)
-    got = oracle.attn_jvp_alg2(Q, K, V, tQ, tK, tV, 1.0, Bc=4)
+    got = oracle.attn_jvp_fold(Q, K, V, tQ, tK, tV, 1.0, Bc=4)
     for u, v in zip(ref, got):
         assert np.abs(u - v).max() <= 1e-11 * (1 + np.abs(u).max())

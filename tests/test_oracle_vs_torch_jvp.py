@@ -23,7 +23,7 @@ def test_vs_torch_func_jvp(oracle, Lq, Lk, D, s):
     want_O, want_tO = torch.func.jvp(lambda a, b, c: _attn(a, b, c, s), (Q, K, V), (tQ, tK, tV))
     want_L, want_mu = torch.func.jvp(lambda a, b: _lse(a, b, s), (Q, K), (tQ, tK))
     for got in (oracle.attn_jvp_def(*[x.numpy() for x in (Q, K, V, tQ, tK, tV)], s),
-                oracle.attn_jvp_alg2(*[x.numpy() for x in (Q, K, V, tQ, tK, tV)], s, Bc=32)):
+                oracle.attn_jvp_fold(*[x.numpy() for x in (Q, K, V, tQ, tK, tV)], s, Bc=32)):
         O, tO, LSE, MU = got
         np.testing.assert_allclose(O, want_O.numpy(), atol=1e-13)
         np.testing.assert_allclose(tO, want_tO.numpy(), atol=1e-13)
