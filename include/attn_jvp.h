@@ -17,7 +17,8 @@
  * Conventions common to every entry point
  *   - All tensor pointers are DEVICE pointers owned by the caller.  The
  *     library neither frees nor retains them and allocates no device memory;
- *     only the split-KV entry point needs a (caller-provided) workspace.
+ *     the split-KV and the host-buffer entry points need a (caller-provided)
+ *     device workspace, all others need none.
  *   - q, tq, o, to : bf16, layout [B][Lq][H][D] contiguous ("BLHD").
  *     k, v, tk, tv : bf16, layout [B][Lk][H][D] contiguous.
  *     lse          : fp32, layout [B][H][Lq], natural log of the scaled scores.
@@ -50,7 +51,7 @@ extern "C" {
 /* error codes */
 #define ATTN_JVP_OK                  0
 #define ATTN_JVP_ERR_NULL            1  /* a required pointer is NULL */
-#define ATTN_JVP_ERR_SHAPE           2  /* B, H, Lq or Lk < 1; B or H > 65535; sizes overflow; bad splits / heads_per_stage */
+#define ATTN_JVP_ERR_SHAPE           2  /* B, H, Lq or Lk < 1; sizes or the work-item count overflow; bad splits / heads_per_stage */
 #define ATTN_JVP_ERR_UNSUPPORTED_D   3  /* D is not 64 or 128 */
 #define ATTN_JVP_ERR_ALIGN           4  /* a tensor pointer is not 16-byte aligned */
 #define ATTN_JVP_ERR_FLAGS           5  /* unknown flag bits */
@@ -167,9 +168,9 @@ int attn_jvp_fwd_host(const void* q, const void* k, const void* v,
  * allowed to allocate GPU memory.  (No counterpart in the paper: this is a packaging variant, the arithmetic
  * is that of attn_jvp_fwd_splitkv.)
  *
- * Who needs it: code that runs where a cudaMalloc is off limits -- inside a region being captured into a CUDA
- * graph or replayed from one, in a real-time or serving loop whose memory was fixed at start-up, under a
- * framework whose allocator must own every byte, or in a process whose memory budget is already spent.  Such
+ * Who needs it: code that runs where a cudaMalloc is off limits -- a real-time or serving loop whose memory was
+ * fixed at start-up and which cannot afford the device-wide synchronisation an allocation implies, a framework
+ * whose allocator must own every byte, or a process whose memory budget is already spent.  Such
  * a caller cannot provide the workspace that attn_jvp_fwd_splitkv asks for, so this entry point brings its own:
  * a fixed array of ATTN_JVP_STATIC_SCRATCH_BYTES (32 MiB) that is part of the library's device image.  Every GPU
  * on which the library is loaded gives up that much memory until the process exits, whether or not this
@@ -184,8 +185,9 @@ int attn_jvp_fwd_host(const void* q, const void* k, const void* v,
  *     returning at once.)
  *   - A call whose chunks need more than ATTN_JVP_STATIC_SCRATCH_BYTES (see attn_jvp_splitkv_workspace_bytes)
  *     is refused with ATTN_JVP_ERR_STATIC_SCRATCH and nothing is enqueued; attn_jvp_strerror gives both sizes.
- *   - The first call on each device looks up the array's device address (with that device current).  Make that
- *     first call outside of any stream capture.
+ *   - The first call on each device looks up the array's device address (with that device current), and the
+ *     first call per (D, flags) combination sets a launch attribute of the kernel it selects.  Make these first
+ *     calls before any stream capture begins.
  *   - All calls on a device share the one array and it keeps whatever the previous call left in it.  Nothing in
  *     it has to start at zero: every value that the merge step reads is written by the same call first.  Two calls
  *     that overlap on the GPU (different streams, no dependency between them) race on the array and produce
@@ -207,8 +209,10 @@ int attn_jvp_set_stream(void* cuda_stream);
  * kernel expired (ATTN_JVP_ERR_DEVICE_LAYOUT if its shared-memory layout did
  * not fit).  Meaningful once the caller has synchronised the stream(s) the
  * kernels ran on; reading it clears it (and lets later launches run again).
- * Copies one word from the device, so it orders itself after work on the
- * legacy default stream; it does not wait for other streams.
+ * Normally this only reads a pinned host word.  It copies a word from the
+ * device (and so orders itself after work on the legacy default stream) only
+ * after a reported timeout, or while attn_jvp_fwd_splitkv_static is the only
+ * entry point that has run on the device; it never waits for other streams.
  */
 int attn_jvp_device_status(void);
 

@@ -151,8 +151,8 @@ def attn_jvp_fwd_splitkv(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, Lk, D, s
 
 def attn_jvp_fwd_splitkv_static(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, Lk, D, scale, flags, splits,
                                 cuda_stream) -> int:
-    """Split-KV for callers that may not allocate GPU memory (inside CUDA-graph capture, fixed-memory serving
-    loops, allocator-owned processes): the chunk partials go to a 32 MiB buffer built into the library instead of
+    """Split-KV for callers that may not allocate GPU memory (serving loops whose memory was fixed at start-up,
+    processes where a framework allocator owns every byte): the chunk partials go to a 32 MiB buffer built into the library instead of
     a caller-provided workspace.  Calls larger than that are refused (ERR_STATIC_SCRATCH); calls that overlap on
     the GPU race on the shared buffer.  Raw call: tensors or device addresses in, return code out."""
     return int(load().attn_jvp_fwd_splitkv_static(_ptr(q), _ptr(k), _ptr(v), _ptr(tq), _ptr(tk), _ptr(tv), _ptr(o),

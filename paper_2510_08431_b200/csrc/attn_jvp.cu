@@ -6,6 +6,7 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
+#include <atomic>
 #include <mutex>
 
 #include "attn_jvp_kernel.cuh"
@@ -23,15 +24,27 @@ thread_local cudaStream_t tl_stream = nullptr;
 thread_local char tl_cuda_msg[256] = "";
 thread_local char tl_strerror_buf[384];
 
-int* g_host_status[kMaxDevices] = {};       // mapped pinned host words, one per device
-int* g_host_status_dev[kMaxDevices] = {};   // their device-side addresses
-int g_sm_count[kMaxDevices] = {};
-int g_dyn_smem[kMaxDevices][2][3][2] = {};  // dynamic shared memory per kernel instantiation, 0 = not set up
-
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn g_encode_tiled = nullptr;
+
+// Lazily initialised per-device state.  Several host threads may make their first call at the same time (the
+// stream of attn_jvp_fwd is per thread): every slow path below runs under `lock`, and what the fast paths read is
+// published through atomics only when complete.
+struct DeviceState {
+    std::mutex lock;
+    std::atomic<int> cc_major{0};                 // 0 = not queried yet
+    int sm_count = 0;                             // valid once cc_major != 0
+    int smem_optin = 0;                           // valid once cc_major != 0
+    std::atomic<int*> host_status{nullptr};       // mapped pinned host word ...
+    std::atomic<int*> host_status_dev{nullptr};   // ... and its device-side address (published first)
+    std::atomic<bool> unwatched_launch{false};    // a kernel ran here before the status word existed
+    std::atomic<int> dyn_smem[2][3][2][2];        // dynamic shared memory per kernel instantiation, 0 = not set up
+    std::atomic<void*> static_scratch{nullptr};   // device address of the built-in scratch array
+};
+DeviceState g_dev[kMaxDevices];
+std::mutex g_encode_lock;
+std::atomic<EncodeTiledFn> g_encode_tiled{nullptr};
 
 int cuda_fail(const char* what, cudaError_t e) {
     snprintf(tl_cuda_msg, sizeof tl_cuda_msg, "%s: %s", what, cudaGetErrorString(e));
@@ -39,7 +52,9 @@ int cuda_fail(const char* what, cudaError_t e) {
 }
 
 int get_encode_fn() {
-    if (g_encode_tiled) return 0;
+    if (g_encode_tiled.load(std::memory_order_acquire)) return 0;
+    std::lock_guard<std::mutex> guard(g_encode_lock);
+    if (g_encode_tiled.load(std::memory_order_relaxed)) return 0;
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
     cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
@@ -48,7 +63,52 @@ int get_encode_fn() {
         snprintf(tl_cuda_msg, sizeof tl_cuda_msg, "cuTensorMapEncodeTiled not available from this driver");
         return ATTN_JVP_ERR_CUDA;
     }
-    g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    g_encode_tiled.store(reinterpret_cast<EncodeTiledFn>(fn), std::memory_order_release);
+    return 0;
+}
+
+// The current device, checked to be sm_100; its attributes are queried once.  Enqueues nothing.
+int current_device(int* dev_out, DeviceState** st_out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail("cudaGetDevice", e);
+    if (dev < 0 || dev >= kMaxDevices) return ATTN_JVP_ERR_ARCH;
+    DeviceState& st = g_dev[dev];
+    if (st.cc_major.load(std::memory_order_acquire) == 0) {
+        std::lock_guard<std::mutex> guard(st.lock);
+        if (st.cc_major.load(std::memory_order_relaxed) == 0) {
+            int major = 0, sms = 0, optin = 0;
+            e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+            if (e != cudaSuccess) return cuda_fail("cudaDeviceGetAttribute(ComputeCapabilityMajor)", e);
+            e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+            if (e != cudaSuccess) return cuda_fail("cudaDeviceGetAttribute(MultiProcessorCount)", e);
+            e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+            if (e != cudaSuccess) return cuda_fail("cudaDeviceGetAttribute(MaxSharedMemoryPerBlockOptin)", e);
+            st.sm_count = sms;
+            st.smem_optin = optin;
+            st.cc_major.store(major > 0 ? major : -1, std::memory_order_release);
+        }
+    }
+    if (st.cc_major.load(std::memory_order_acquire) != 10) return ATTN_JVP_ERR_ARCH;
+    *dev_out = dev;
+    *st_out = &st;
+    return 0;
+}
+
+// The pinned status word a kernel writes its timeout code to; allocated on the first call that may allocate.
+int ensure_status_word(DeviceState& st) {
+    if (st.host_status.load(std::memory_order_acquire)) return 0;
+    std::lock_guard<std::mutex> guard(st.lock);
+    if (st.host_status.load(std::memory_order_relaxed)) return 0;
+    int* hp = nullptr;
+    cudaError_t e = cudaHostAlloc((void**)&hp, sizeof(int), cudaHostAllocMapped);
+    if (e != cudaSuccess) return cuda_fail("cudaHostAlloc(status word)", e);
+    *hp = 0;
+    int* dp = nullptr;
+    e = cudaHostGetDevicePointer((void**)&dp, hp, 0);
+    if (e != cudaSuccess) { cudaFreeHost(hp); return cuda_fail("cudaHostGetDevicePointer", e); }
+    st.host_status_dev.store(dp, std::memory_order_release);   // a reader that sees the host pointer sees this one too
+    st.host_status.store(hp, std::memory_order_release);
     return 0;
 }
 
@@ -59,7 +119,7 @@ int make_map(CUtensorMap* map, const void* base, int B, int L, int H, int D, int
     const cuuint64_t strides[3] = {(cuuint64_t)D * 2, (cuuint64_t)H * D * 2, (cuuint64_t)L * H * D * 2};
     const cuuint32_t box[4] = {64, 1, (cuuint32_t)rows, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
+    CUresult r = g_encode_tiled.load(std::memory_order_acquire)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -76,29 +136,32 @@ bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
 }
 
 template <int D, int MODE, bool SPLIT>
-int launch(const CUtensorMap* maps, const KernelArgs& ka, dim3 grid, cudaStream_t stream, int dev) {
+int launch(const CUtensorMap* maps, const KernelArgs& ka, dim3 grid, cudaStream_t stream, DeviceState& st) {
     auto kern = attn_jvp::attn_jvp_fwd_kernel<D, MODE, SPLIT>;
-    int& smem = g_dyn_smem[dev][D == 128][MODE][SPLIT];
+    std::atomic<int>& slot = st.dyn_smem[D == 128][MODE][SPLIT][0];
+    int smem = slot.load(std::memory_order_acquire);
     if (smem == 0) {
         // dynamic shared memory = the operand layout plus slack for its 1024-byte alignment, capped by
         // what the device leaves after the kernel's static shared memory
-        cudaFuncAttributes fa;
-        cudaError_t e = cudaFuncGetAttributes(&fa, kern);
-        if (e != cudaSuccess) return cuda_fail("cudaFuncGetAttributes", e);
-        int optin = 0;
-        e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-        if (e != cudaSuccess) return cuda_fail("cudaDeviceGetAttribute(MaxSharedMemoryPerBlockOptin)", e);
-        int want = attn_jvp::SmemPlan<D>::kDynBytes;
-        const int room = optin - (int)fa.sharedSizeBytes;
-        if (want > room) want = room;
-        if (want < attn_jvp::SmemPlan<D>::kBytes) {
-            snprintf(tl_cuda_msg, sizeof tl_cuda_msg, "device offers %d bytes of shared memory, kernel needs %d",
-                     room, attn_jvp::SmemPlan<D>::kBytes);
-            return ATTN_JVP_ERR_CUDA;
+        std::lock_guard<std::mutex> guard(st.lock);
+        smem = slot.load(std::memory_order_relaxed);
+        if (smem == 0) {
+            cudaFuncAttributes fa;
+            cudaError_t e = cudaFuncGetAttributes(&fa, kern);
+            if (e != cudaSuccess) return cuda_fail("cudaFuncGetAttributes", e);
+            int want = attn_jvp::SmemPlan<D>::kDynBytes;
+            const int room = st.smem_optin - (int)fa.sharedSizeBytes;
+            if (want > room) want = room;
+            if (want < attn_jvp::SmemPlan<D>::kBytes) {
+                snprintf(tl_cuda_msg, sizeof tl_cuda_msg, "device offers %d bytes of shared memory, kernel needs %d",
+                         room, attn_jvp::SmemPlan<D>::kBytes);
+                return ATTN_JVP_ERR_CUDA;
+            }
+            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, want);
+            if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
+            smem = want;
+            slot.store(want, std::memory_order_release);
         }
-        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, want);
-        if (e != cudaSuccess) return cuda_fail("cudaFuncSetAttribute(MaxDynamicSharedMemorySize)", e);
-        smem = want;
     }
     kern<<<grid, attn_jvp::kThreads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], maps[6],
                                                      maps[7], ka);
@@ -140,7 +203,6 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     const int mode = fwd_only ? attn_jvp::kModeFwdOnly : (kv_free ? attn_jvp::kModeKvTangentFree : attn_jvp::kModeJvp);
     if (B < 1 || H < 1 || Lq < 1 || Lk < 1) return ATTN_JVP_ERR_SHAPE;
     if (D != 64 && D != 128) return ATTN_JVP_ERR_UNSUPPORTED_D;
-    if (B > 65535 || H > 65535) return ATTN_JVP_ERR_SHAPE;   // documented limits of the interface
     const long double nq = (long double)B * H * Lq * D, nk = (long double)B * H * Lk * D;
     if (nq * 2 > 9.0e18L || nk * 2 > 9.0e18L) return ATTN_JVP_ERR_SHAPE;
     if (!q || !k || !v || !o || !lse) return ATTN_JVP_ERR_NULL;
@@ -151,12 +213,16 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     int tiles_per_split = 0, eff_splits = 1;
     split_plan(Lk, splits, &tiles_per_split, &eff_splits);
     const bool split = eff_splits > 1;
+    // work items = query tiles x heads x batch x chunks; item + gridDim.x must not overflow an int in the kernel
+    const long long n_q_tiles = (Lq + attn_jvp::kBlockM - 1) / attn_jvp::kBlockM;
+    const long double n_items_ld = (long double)n_q_tiles * H * B * eff_splits;
+    if (n_items_ld > (long double)(0x7fffffffLL - 65536)) return ATTN_JVP_ERR_SHAPE;
+    const long long n_items = n_q_tiles * H * B * eff_splits;
     SplitLayout lay = split_layout(B, H, Lq, D, eff_splits);
     if (split) {
         if (!workspace) return ATTN_JVP_ERR_NULL;
         if ((uintptr_t)workspace & 15u) return ATTN_JVP_ERR_ALIGN;
         if (workspace_bytes < lay.total) return ATTN_JVP_ERR_WORKSPACE;
-        if ((long long)B * eff_splits > 65535) return ATTN_JVP_ERR_SHAPE;
     }
     const void* used_in[6] = {q, k, v, fwd_only ? nullptr : tq, mode == attn_jvp::kModeJvp ? tk : nullptr,
                               mode == attn_jvp::kModeJvp ? tv : nullptr};
@@ -175,26 +241,14 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     }
 
     int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return cuda_fail("cudaGetDevice", e);
-    if (dev < 0 || dev >= kMaxDevices) return ATTN_JVP_ERR_ARCH;
-    int major = 0;
-    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
-    if (e != cudaSuccess) return cuda_fail("cudaDeviceGetAttribute", e);
-    if (major != 10) return ATTN_JVP_ERR_ARCH;
-
+    DeviceState* stp = nullptr;
+    if (int rc = current_device(&dev, &stp)) return rc;
+    DeviceState& st = *stp;
     if (int rc = get_encode_fn()) return rc;
-    if (!g_host_status[dev] && may_allocate) {
-        int* hp = nullptr;
-        e = cudaHostAlloc((void**)&hp, sizeof(int), cudaHostAllocMapped);
-        if (e != cudaSuccess) return cuda_fail("cudaHostAlloc(status word)", e);
-        *hp = 0;
-        int* dp = nullptr;
-        e = cudaHostGetDevicePointer((void**)&dp, hp, 0);
-        if (e != cudaSuccess) { cudaFreeHost(hp); return cuda_fail("cudaHostGetDevicePointer", e); }
-        g_host_status[dev] = hp;
-        g_host_status_dev[dev] = dp;
+    if (may_allocate) {
+        if (int rc = ensure_status_word(st)) return rc;
     }
+    cudaError_t e;
 
     // ---- tensor maps (Q-side boxes are 128 rows, K-side boxes 64 rows) ----
     CUtensorMap maps[8];
@@ -212,7 +266,9 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     ka.o = reinterpret_cast<__nv_bfloat16*>(o);
     ka.to = reinterpret_cast<__nv_bfloat16*>(to);
     ka.lse = lse;
-    ka.host_status = g_host_status_dev[dev];   // null if no call on this device was allowed to allocate it yet
+    ka.host_status = st.host_status_dev.load(std::memory_order_acquire);
+    // no status word yet (only the allocation-free entry point has run here): the device-side flag is the only record
+    if (ka.host_status == nullptr) st.unwatched_launch.store(true, std::memory_order_release);
     ka.H = H;
     ka.Lq = Lq;
     ka.Lk = Lk;
@@ -233,31 +289,22 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     }
 
     // persistent CTAs: one per SM (fewer if there is less work), sharing the work items round-robin
-    const long long n_q_tiles = (Lq + attn_jvp::kBlockM - 1) / attn_jvp::kBlockM;
-    const long long n_items = n_q_tiles * H * B * eff_splits;
-    if (n_items > 0x7fffffffLL - 65536) return ATTN_JVP_ERR_SHAPE;   // item + gridDim.x must not overflow an int
     ka.n_q_tiles = (int)n_q_tiles;
     ka.n_items = (int)n_items;
-    if (g_sm_count[dev] == 0) {
-        int sms = 0;
-        e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return cuda_fail("cudaDeviceGetAttribute(MultiProcessorCount)", e);
-        g_sm_count[dev] = sms;
-    }
     // Short items (few key tiles): one persistent CTA per SM, so that the epilogue of an item overlaps the
     // start of the next.  Long items: one CTA per item, which lets the hardware balance the load (a static
     // round-robin costs up to one item of imbalance at the end, which is more than the overlap saves there).
     const int tiles_per_item = split ? tiles_per_split : ka.n_kv_tiles;
     const bool persistent = tiles_per_item <= kPersistentMaxTiles;
-    const long long n_ctas = (persistent && n_items > g_sm_count[dev]) ? g_sm_count[dev] : n_items;
+    const long long n_ctas = (persistent && n_items > st.sm_count) ? st.sm_count : n_items;
     const dim3 grid((unsigned)n_ctas, 1, 1);
     int rc;
 #define ATTN_JVP_DISPATCH(DD, SS)                                                                                  \
     switch (mode) {                                                                                               \
-        case attn_jvp::kModeJvp: rc = launch<DD, attn_jvp::kModeJvp, SS>(maps, ka, grid, stream, dev); break;      \
+        case attn_jvp::kModeJvp: rc = launch<DD, attn_jvp::kModeJvp, SS>(maps, ka, grid, stream, st); break;      \
         case attn_jvp::kModeKvTangentFree:                                                                        \
-            rc = launch<DD, attn_jvp::kModeKvTangentFree, SS>(maps, ka, grid, stream, dev); break;                 \
-        default: rc = launch<DD, attn_jvp::kModeFwdOnly, SS>(maps, ka, grid, stream, dev); break;                  \
+            rc = launch<DD, attn_jvp::kModeKvTangentFree, SS>(maps, ka, grid, stream, st); break;                 \
+        default: rc = launch<DD, attn_jvp::kModeFwdOnly, SS>(maps, ka, grid, stream, st); break;                  \
     }
     if (D == 128) {
         if (split) { ATTN_JVP_DISPATCH(128, true) } else { ATTN_JVP_DISPATCH(128, false) }
@@ -295,19 +342,28 @@ struct HostPipe {
 };
 HostPipe g_host_pipe[kMaxDevices];
 
+// Creates the pipeline's streams and events; on failure everything created so far is released again.
 int host_pipe_setup(HostPipe& hp) {
     if (hp.ready) return 0;
-    cudaError_t e;
     cudaStream_t* streams[3] = {&hp.in, &hp.comp, &hp.out};
-    for (cudaStream_t* st : streams) {
-        e = cudaStreamCreateWithFlags(st, cudaStreamNonBlocking);
-        if (e != cudaSuccess) return cuda_fail("cudaStreamCreateWithFlags", e);
-    }
     cudaEvent_t* events[10] = {&hp.start, &hp.in_done[0], &hp.in_done[1], &hp.comp_done[0], &hp.comp_done[1],
                                &hp.out_done[0], &hp.out_done[1], &hp.end_in, &hp.end_comp, &hp.end_out};
+    cudaError_t e = cudaSuccess;
+    const char* what = nullptr;
+    for (cudaStream_t* st : streams) {
+        if (e != cudaSuccess) break;
+        e = cudaStreamCreateWithFlags(st, cudaStreamNonBlocking);
+        if (e != cudaSuccess) { *st = nullptr; what = "cudaStreamCreateWithFlags"; }
+    }
     for (cudaEvent_t* ev : events) {
+        if (e != cudaSuccess) break;
         e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming);
-        if (e != cudaSuccess) return cuda_fail("cudaEventCreateWithFlags", e);
+        if (e != cudaSuccess) { *ev = nullptr; what = "cudaEventCreateWithFlags"; }
+    }
+    if (e != cudaSuccess) {
+        for (cudaEvent_t* ev : events) if (*ev) { cudaEventDestroy(*ev); *ev = nullptr; }
+        for (cudaStream_t* st : streams) if (*st) { cudaStreamDestroy(*st); *st = nullptr; }
+        return cuda_fail(what, e);
     }
     hp.ready = true;
     return 0;
@@ -346,7 +402,6 @@ int run_host(const void* q, const void* k, const void* v, const void* tq, const 
     const bool jvp_kv = !fwd_only && (flags & ATTN_JVP_KV_TANGENT_FREE) == 0;
     if (B < 1 || H < 1 || Lq < 1 || Lk < 1 || heads_per_stage < 0) return ATTN_JVP_ERR_SHAPE;
     if (D != 64 && D != 128) return ATTN_JVP_ERR_UNSUPPORTED_D;
-    if (B > 65535 || H > 65535) return ATTN_JVP_ERR_SHAPE;
     const long double nq_all = (long double)B * H * Lq * D, nk_all = (long double)B * H * Lk * D;
     if (nq_all * 2 > 9.0e18L || nk_all * 2 > 9.0e18L) return ATTN_JVP_ERR_SHAPE;
     if (!q || !k || !v || !o || !lse || !workspace) return ATTN_JVP_ERR_NULL;
@@ -358,28 +413,28 @@ int run_host(const void* q, const void* k, const void* v, const void* tq, const 
     const HostLayout lay = host_layout(B, Lq, Lk, D, hg);
     if (workspace_bytes < lay.total) return ATTN_JVP_ERR_WORKSPACE;
 
+    // everything that can refuse the call without touching a stream comes first: nothing is enqueued on error
     int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return cuda_fail("cudaGetDevice", e);
-    if (dev < 0 || dev >= kMaxDevices) return ATTN_JVP_ERR_ARCH;
+    DeviceState* stp = nullptr;
+    if (int rc = current_device(&dev, &stp)) return rc;
+    if (int rc = get_encode_fn()) return rc;
+    if (int rc = ensure_status_word(*stp)) return rc;
     HostPipe& hp = g_host_pipe[dev];
     std::lock_guard<std::mutex> guard(hp.lock);
     if (int rc = host_pipe_setup(hp)) return rc;
-
-    // everything below runs after what the caller has already put on `stream` ...
-    e = cudaEventRecord(hp.start, stream);
-    if (e != cudaSuccess) return cuda_fail("cudaEventRecord", e);
-    cudaStream_t internal[3] = {hp.in, hp.comp, hp.out};
-    for (cudaStream_t st : internal) {
-        e = cudaStreamWaitEvent(st, hp.start, 0);
-        if (e != cudaSuccess) return cuda_fail("cudaStreamWaitEvent", e);
-    }
 
     const size_t row_host = (size_t)H * D * 2;      // bytes between consecutive (b, l) rows of a host tensor
     int rc = 0;
     cudaError_t ce = cudaSuccess;
     const char* what = nullptr;
     auto check = [&](cudaError_t err, const char* w) { if (err != cudaSuccess && ce == cudaSuccess) { ce = err; what = w; } };
+
+    // everything below runs after what the caller has already put on `stream` ...
+    cudaError_t e = cudaEventRecord(hp.start, stream);
+    if (e != cudaSuccess) return cuda_fail("cudaEventRecord", e);
+    cudaStream_t internal[3] = {hp.in, hp.comp, hp.out};
+    for (cudaStream_t st : internal) check(cudaStreamWaitEvent(st, hp.start, 0), "cudaStreamWaitEvent");
+
     const int n_stages = (H + hg - 1) / hg;
     for (int g = 0; g < n_stages && rc == 0 && ce == cudaSuccess; ++g) {
         const int set = g & 1;
@@ -433,7 +488,8 @@ int run_host(const void* q, const void* k, const void* v, const void* tq, const 
               "cudaMemcpy2DAsync (LSE)");
         check(cudaEventRecord(hp.out_done[set], hp.out), "cudaEventRecord");
     }
-    // ... and the caller's stream continues after all of it (also when an error cut the loop short)
+    // ... and the caller's stream continues after all of it (also when an error cut the loop short: the internal
+    // streams are never left chained to the caller's stream without the closing join)
     check(cudaEventRecord(hp.end_in, hp.in), "cudaEventRecord");
     check(cudaEventRecord(hp.end_comp, hp.comp), "cudaEventRecord");
     check(cudaEventRecord(hp.end_out, hp.out), "cudaEventRecord");
@@ -518,7 +574,6 @@ int attn_jvp_fwd_host(const void* q, const void* k, const void* v, const void* t
 // Scratch for callers that cannot allocate: lives in the library's device image, so every GPU that loads
 // the library holds these bytes until the process exits.
 static __device__ __align__(256) unsigned char g_static_scratch[ATTN_JVP_STATIC_SCRATCH_BYTES];
-static void* g_static_scratch_dev[kMaxDevices] = {};   // device address of the array, looked up once per device
 
 int attn_jvp_fwd_splitkv_static(const void* q, const void* k, const void* v, const void* tq, const void* tk,
                                 const void* tv, void* o, void* to, float* lse, float* mu, int B, int H, int Lq, int Lk,
@@ -532,18 +587,21 @@ int attn_jvp_fwd_splitkv_static(const void* q, const void* k, const void* v, con
         return ATTN_JVP_ERR_STATIC_SCRATCH;
     }
     int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return cuda_fail("cudaGetDevice", e);
-    if (dev < 0 || dev >= kMaxDevices) return ATTN_JVP_ERR_ARCH;
-    if (!g_static_scratch_dev[dev]) {
+    DeviceState* stp = nullptr;
+    if (int rc = current_device(&dev, &stp)) return rc;
+    void* scratch = stp->static_scratch.load(std::memory_order_acquire);
+    if (!scratch) {
         // In host code the array's name only stands for the symbol; its address on the current device has to be
-        // asked for.  Done once per device, on the first call (which should therefore precede any stream capture).
-        void* p = nullptr;
-        e = cudaGetSymbolAddress(&p, g_static_scratch);
-        if (e != cudaSuccess) return cuda_fail("cudaGetSymbolAddress(static scratch)", e);
-        g_static_scratch_dev[dev] = p;
+        // asked for.  Done once per device, on the first call here.
+        std::lock_guard<std::mutex> guard(stp->lock);
+        scratch = stp->static_scratch.load(std::memory_order_relaxed);
+        if (!scratch) {
+            cudaError_t e = cudaGetSymbolAddress(&scratch, g_static_scratch);
+            if (e != cudaSuccess) return cuda_fail("cudaGetSymbolAddress(static scratch)", e);
+            stp->static_scratch.store(scratch, std::memory_order_release);
+        }
     }
-    return run(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, Lk, D, scale, flags, splits, g_static_scratch_dev[dev],
+    return run(q, k, v, tq, tk, tv, o, to, lse, mu, B, H, Lq, Lk, D, scale, flags, splits, scratch,
                (size_t)ATTN_JVP_STATIC_SCRATCH_BYTES, static_cast<cudaStream_t>(cuda_stream), /*may_allocate=*/false);
 }
 
@@ -562,11 +620,10 @@ int attn_jvp_qknorm_fwd(const void* x, const void* tx, const float* w, void* y, 
         overlaps(ty, bytes, w, (size_t)D * 4))
         return ATTN_JVP_ERR_ALIAS;
     int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return cuda_fail("cudaGetDevice", e);
-    int sms = 0;
-    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    if (e != cudaSuccess) return cuda_fail("cudaDeviceGetAttribute(MultiProcessorCount)", e);
+    DeviceState* stp = nullptr;
+    if (int rc = current_device(&dev, &stp)) return rc;
+    const int sms = stp->sm_count;
+    cudaError_t e;
     const int rows_per_block = 256 / (D / 8);
     long long blocks = (rows + rows_per_block - 1) / rows_per_block;
     const long long cap = (long long)sms * 16;                 // a multiple of the SM count; the kernel strides
@@ -590,15 +647,12 @@ int attn_jvp_qknorm_fwd(const void* x, const void* tx, const float* w, void* y, 
 
 int attn_jvp_selftest_bounded_wait(void* cuda_stream) {
     int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return cuda_fail("cudaGetDevice", e);
-    if (dev < 0 || dev >= kMaxDevices) return ATTN_JVP_ERR_ARCH;
-    int major = 0;
-    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
-    if (e != cudaSuccess) return cuda_fail("cudaDeviceGetAttribute", e);
-    if (major != 10) return ATTN_JVP_ERR_ARCH;
-    attn_jvp::bounded_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(g_host_status_dev[dev]);
-    e = cudaGetLastError();
+    DeviceState* stp = nullptr;
+    if (int rc = current_device(&dev, &stp)) return rc;
+    if (int rc = ensure_status_word(*stp)) return rc;
+    attn_jvp::bounded_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+        stp->host_status_dev.load(std::memory_order_acquire));
+    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail("self-test kernel launch", e);
     return 0;
 }
@@ -611,19 +665,27 @@ int attn_jvp_set_stream(void* cuda_stream) {
 int attn_jvp_device_status(void) {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    DeviceState& ds = g_dev[dev];
     int st = 0;
-    int* hp = g_host_status[dev];
+    int* hp = ds.host_status.load(std::memory_order_acquire);
     if (hp) {
         st = *reinterpret_cast<volatile int*>(hp);
         if (st != 0) *reinterpret_cast<volatile int*>(hp) = 0;
     }
-    // The kernels also raise a device-side flag (later launches test it and return at once).  It is the only
-    // record when no status word exists yet, i.e. when only the allocation-free entry point has run here.
-    int flag = 0;
-    if (cudaMemcpyFromSymbol(&flag, attn_jvp::g_abort_flag, sizeof(int)) == cudaSuccess && flag != 0) {
-        if (st == 0) st = ATTN_JVP_ERR_DEVICE_TIMEOUT;
-        const int zero = 0;
-        cudaMemcpyToSymbol(attn_jvp::g_abort_flag, &zero, sizeof(int));   // let later launches run again
+    // The kernels also raise a device-side flag (later launches test it and return at once).  Reading it is a
+    // blocking copy, so it is read only when it can hold news: a timeout was just reported through the status
+    // word (then it has to be cleared), or kernels ran here before the status word existed (then it is the only
+    // record, which is the case when only the allocation-free entry point has been used).
+    if (st != 0 || ds.unwatched_launch.load(std::memory_order_acquire)) {
+        int flag = 0;
+        if (cudaMemcpyFromSymbol(&flag, attn_jvp::g_abort_flag, sizeof(int)) == cudaSuccess) {
+            if (flag != 0) {
+                if (st == 0) st = ATTN_JVP_ERR_DEVICE_TIMEOUT;
+                const int zero = 0;
+                cudaMemcpyToSymbol(attn_jvp::g_abort_flag, &zero, sizeof(int));   // let later launches run again
+            }
+            if (hp) ds.unwatched_launch.store(false, std::memory_order_release);
+        }
     }
     return st;
 }
@@ -632,7 +694,7 @@ const char* attn_jvp_strerror(int code) {
     switch (code) {
         case ATTN_JVP_OK: return "ok";
         case ATTN_JVP_ERR_NULL: return "a required pointer is NULL";
-        case ATTN_JVP_ERR_SHAPE: return "B, H, Lq and Lk must be >= 1 (B, H <= 65535) and sizes must not overflow";
+        case ATTN_JVP_ERR_SHAPE: return "B, H, Lq and Lk must be >= 1 and the tensor sizes and the number of work items must not overflow";
         case ATTN_JVP_ERR_UNSUPPORTED_D: return "head dimension D must be 64 or 128";
         case ATTN_JVP_ERR_ALIGN: return "tensor pointers must be 16-byte aligned";
         case ATTN_JVP_ERR_FLAGS: return "unknown flag bits";

@@ -58,6 +58,9 @@ WORKLOADS = {
     # not one of the five benchmark configs: few queries against a long key sequence, the case the
     # split-KV entry point exists for (32 query tiles x heads CTAs would fill a fifth of the GPU)
     "few_q_long_k": Workload("few_q_long_k", 1, 8, 512, 32760, 128, 1.0, 0.5, 5),
+    # head dimension 64 (the library's other supported D) at the image and the video sequence lengths
+    "image_dit_d64": Workload("image_dit_d64", 2, 24, 4096, 4096, 64, 1.0, 0.5, 6),
+    "video_dit_d64": Workload("video_dit_d64", 1, 24, 32760, 32760, 64, 1.0, 0.5, 7),
 }
 
 

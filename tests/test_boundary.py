@@ -61,7 +61,8 @@ def _args(**kw):
 
 @pytest.mark.parametrize("kw,code", [
     (dict(flags=4), 5), (dict(flags=0x80000000), 5),
-    (dict(B=0), 2), (dict(H=0), 2), (dict(Lq=0), 2), (dict(Lk=0), 2), (dict(Lk=-3), 2), (dict(H=70000), 2),
+    (dict(B=0), 2), (dict(H=0), 2), (dict(Lq=0), 2), (dict(Lk=0), 2), (dict(Lk=-3), 2),
+    (dict(B=1 << 20, H=1 << 20, Lq=1, Lk=1), 2),       # more work items than the kernel can index
     (dict(D=96), 3), (dict(D=0), 3), (dict(D=256), 3),
     (dict(q=None), 1), (dict(k=None), 1), (dict(v=None), 1), (dict(o=None), 1), (dict(lse=None), 1),
     (dict(tq=None), 1), (dict(to=None), 1), (dict(tk=None), 1), (dict(tv=None), 1),
@@ -73,6 +74,31 @@ def _args(**kw):
 ])
 def test_bad_arguments_are_rejected_before_any_gpu_work(lib, kw, code):
     assert lib.attn_jvp_fwd(**_args(**kw)) == code
+
+
+def test_concurrent_first_calls_from_two_threads(lib):
+    """The library's per-device state is set up lazily; two host threads whose first calls race must both come
+    back with a clean return code.  Fake addresses: without a CUDA device the calls pass validation and stop at
+    the device check, which is the lazily initialised part that can be reached here."""
+    import threading
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("would enqueue work on fake addresses")
+    codes = [None] * 8
+    gate = threading.Barrier(len(codes))
+
+    def first_call(i):
+        gate.wait()
+        codes[i] = lib.attn_jvp_fwd(**_args()) if i % 2 == 0 else lib.attn_jvp_qknorm_fwd(
+            A, A + STEP, A + 2 * STEP, A + 3 * STEP, A + 4 * STEP, 64, 64, 1e-6, None)
+
+    threads = [threading.Thread(target=first_call, args=(i,)) for i in range(len(codes))]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert all(c in (8, 9) for c in codes), codes   # ERR_ARCH / ERR_CUDA: no device; nothing crashed or hung
+    assert lib.attn_jvp_device_status() == 0
 
 
 def test_ignored_pointers_may_be_null_or_aliased(lib):

@@ -1,7 +1,8 @@
 """The allocation-free split-KV entry point (attn_jvp_fwd_splitkv_static) against the workspace-taking one.
 
-Some callers may not allocate GPU memory at all: code running inside CUDA-graph capture or replay, serving
-loops whose memory was fixed at start-up, processes where a framework allocator owns every byte.  For them the
+Some callers may not allocate GPU memory at all: serving loops whose memory was fixed at start-up and which
+cannot take the device-wide synchronisation of an allocation, processes where a framework allocator owns every
+byte.  For them the
 library carries a 32 MiB scratch buffer of its own.  This file is collected last on purpose, so that a run that
 stops at the first failure has already been through every other test; it also passes when run alone in a fresh
 process (then its first call is the very first use of the library on the device).
@@ -68,6 +69,31 @@ def test_static_scratch_matches_workspace_version_twice_in_a_row(aj):
     _both_ways(aj, (1, 4, 300, 2000, 128), splits=4, seed=70)
     _both_ways(aj, (2, 2, 130, 700, 64), splits=3, seed=71, flags=aj.KV_TANGENT_FREE)
     _both_ways(aj, (1, 4, 300, 2000, 128), splits=4, seed=72)
+
+
+def test_static_call_leaves_device_memory_in_use_unchanged(aj):
+    """What the entry point is for, observed rather than read from its source: after one warm-up call (module
+    loading and the address look-up happen there) the free device memory reported by the driver is the same
+    before and after a call."""
+    B, H, Lq, Lk, D, splits = 1, 4, 300, 2000, 128, 4
+    x = synth.make_inputs(B, H, Lq, Lk, D, 1.0, 0.5, seed=73)
+    g = {k: t.cuda() for k, t in x.items()}
+    o, to, lse, mu = _buffers(B, H, Lq, D, 0.0)
+    stream = torch.cuda.current_stream().cuda_stream
+
+    def call():
+        rc = aj.attn_jvp_fwd_splitkv_static(g["q"], g["k"], g["v"], g["tq"], g["tk"], g["tv"], o, to, lse, mu,
+                                            B, H, Lq, Lk, D, D ** -0.5, 0, splits, stream)
+        assert rc == 0, aj.attn_jvp_strerror(rc)
+        torch.cuda.synchronize()
+
+    call()
+    free_before, _ = torch.cuda.mem_get_info()
+    call()
+    call()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before, (free_before, free_after)
+    assert aj.attn_jvp_device_status() == 0
 
 
 def test_static_scratch_refuses_oversized_calls(aj):
