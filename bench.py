@@ -39,9 +39,17 @@ FALLBACK_BF16_TFLOPS = 1590.0   # earlier measurement on this machine, used only if
 DATASHEET_BF16_TFLOPS = 2250.0
 
 # DRAM bytes per launch of attn_jvp_fwd_kernel<128, jvp> measured with ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum) on the image_dit_2b workload, see profiles/; scaled to other workloads by their
-# algorithmic bytes (traffic is proportional to the tensors streamed once from HBM; K/V re-reads hit L2).
-NCU_TRAFFIC_BYTES = {"workload": "image_dit_2b", "bytes": 250.1e6}   # 203.0 MB read + 47.1 MB written (mean of two launches)
+# dram__bytes_write.sum), see profiles/.  One capture per sequence-length class: whether the K/V re-reads of a
+# head stay in L2 depends on the sequence length, so a workload takes the capture of its own class and scales it
+# by algorithmic bytes (within a class traffic is proportional to the tensors streamed once from HBM).
+NCU_TRAFFIC_BYTES = {
+    "short": {"workload": "image_dit_2b", "bytes": 250.1e6},     # L = 4096: 203.0 MB read + 47.1 MB written
+    "long": {"workload": "image_dit_2b", "bytes": 250.1e6},      # L = 32760: replaced by its own capture when there is one
+}
+
+
+def traffic_class(w) -> str:
+    return "long" if w.Lk > 8192 else "short"
 
 
 def algorithmic_bytes(w) -> int:
@@ -157,7 +165,8 @@ def run_reference(args, w):
             times.append(res["seconds"]); rows += res["rows"]
     total = sum(times)
     value = rows * 12 * w.Lk * w.D / total / 1e12
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+            "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": workload_config(w, extra={"reference": "fp64 CPU oracle; each step a bounded row sample"}),
@@ -231,6 +240,94 @@ def workload_config(w, extra=None):
     return cfg
 
 
+def run_cp_ranks(args, w, aj):
+    """--cp P with P ranks: one step = exchange the sequence slices all-to-all, run the kernel on this rank's H/P
+    heads over the whole sequence, exchange O, tO, LSE back (strong scaling: the workload is fixed, the ranks
+    share it).  Time = max over ranks; value = the whole workload's flops over it."""
+    import torch.distributed as dist
+    from paper_2510_08431_b200.ulysses import UlyssesAttentionJVP
+    rank, local_rank, P = int(os.environ["RANK"]), int(os.environ.get("LOCAL_RANK", "0")), args.cp
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist.init_process_group("nccl", device_id=dev)
+    if w.Lq % P or w.Lk % P or w.H % P:
+        raise RuntimeError(f"--cp {P} needs Lq, Lk and H to be multiples of {P}")
+    # this rank's sequence slices, all heads; a replicated constant context for the tangent-free workload
+    xs = synth.make_inputs(w.B, w.H, w.Lq // P, w.Lk if w.kv_tangent_free else w.Lk // P, w.D, w.sigma_primal,
+                           w.sigma_tangent, w.seed + (0 if w.kv_tangent_free else 1000 * rank), w.kv_tangent_free,
+                           pin_memory=True)
+    if w.kv_tangent_free:   # queries differ per rank, the context does not
+        xq = synth.make_inputs(w.B, w.H, w.Lq // P, 1, w.D, w.sigma_primal, w.sigma_tangent, w.seed + 1000 * rank + 1,
+                               True, pin_memory=True)
+        xs["q"], xs["tq"] = xq["q"], xq["tq"]
+    g = {k: (None if t is None else t.to(dev)) for k, t in xs.items()}
+    layer = UlyssesAttentionJVP(scale=w.scale)
+    stream = torch.cuda.current_stream()
+
+    def step(x):
+        return layer(x["q"], x["k"], x["v"], x["tq"], x["tk"], x["tv"], kv_replicated=w.kv_tangent_free)
+
+    def bracket(fn, n):
+        dist.barrier(); torch.cuda.synchronize()
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(n):
+            fn()
+        b.record(stream)
+        dist.barrier(); torch.cuda.synchronize()
+        return replicas.max_over_ranks(a.elapsed_time(b), dist, dev) / n
+
+    for _ in range(args.warmup):
+        step(g)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ms = bracket(lambda: step(g), args.steps)
+    clocks = sampler.stop() if rank == 0 else None
+
+    # end to end: pinned host slices in, results out to pinned host memory, every step
+    ho = torch.empty(xs["q"].shape, dtype=torch.bfloat16, pin_memory=True)
+    hto = torch.empty_like(ho).pin_memory()
+    hl = torch.empty((w.B, w.H, w.Lq // P), dtype=torch.float32, pin_memory=True)
+
+    def e2e_step():
+        x = {k: (None if t is None else t.to(dev, non_blocking=True)) for k, t in xs.items()}
+        o, to, lse = step(x)
+        ho.copy_(o, non_blocking=True); hto.copy_(to, non_blocking=True); hl.copy_(lse, non_blocking=True)
+
+    e2e_step()
+    n_e2e = max(2, min(args.steps, 5))
+    e2e_ms = bracket(e2e_step, n_e2e)
+    st = aj.attn_jvp_device_status()
+    if st != 0:
+        raise RuntimeError(aj.attn_jvp_strerror(st))
+    if rank == 0:
+        h2d = sum(t.numel() * 2 for t in xs.values() if t is not None)
+        d2h = ho.numel() * 4 + hl.numel() * 4
+        line = {"metric": METRIC, "value": w.flops / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": P,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+                "scaling": "strong", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "config": workload_config(w, extra={"parallelism": f"ulysses context parallel, P = {P}: all-to-all "
+                                                    "of the inputs, kernel on H/P heads, all-to-all of the outputs"}),
+                "clocks": clocks,
+                "e2e": {"value": w.flops / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                        "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": n_e2e},
+                "gpu_launches": args.steps, "roofline": None}
+        print(json.dumps(line), flush=True)
+    dist.destroy_process_group()
+
+
+def relaunch_with_ranks(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: start N ranks of this script under torchrun and wait."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -243,9 +340,22 @@ def main():
     ap.add_argument("--splits", type=int, default=1, help="key chunks (split-KV entry point) for few-query workloads")
     ap.add_argument("--op", default="attention", choices=["attention", "qknorm"],
                     help="attention = the hot path (default); qknorm = the RMS-norm JVP that feeds it (memory bound)")
+    ap.add_argument("--cp", type=int, default=1,
+                    help="Ulysses context-parallel size P: every rank's call covers H/P heads and the whole sequence "
+                         "(the paper trains the 14B video model with P = 10, i.e. 4 heads per GPU and call).  With "
+                         "P ranks launched (--gpus P) the all-to-all exchange of the six inputs and of O, tO, LSE is "
+                         "inside the timed step; with one rank only the per-rank kernel shape is timed")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     w = synth.WORKLOADS[args.workload]
+
+    world_env = os.environ.get("WORLD_SIZE")
+    if args.impl == "ours" and args.gpus > 1 and world_env is None:
+        if not torch.cuda.is_available() or torch.cuda.device_count() < args.gpus:
+            raise RuntimeError(f"--gpus {args.gpus} needs that many CUDA devices on this node")
+        sys.exit(relaunch_with_ranks(args.gpus))
+    if world_env is not None and int(world_env) != args.gpus:
+        raise RuntimeError(f"--gpus {args.gpus} does not match the {world_env} ranks that were launched")
 
     if args.impl == "reference":
         run_reference(args, w)
@@ -256,6 +366,18 @@ def main():
     if args.op == "qknorm":
         run_qknorm(args, w, aj)
         return
+    cp_note = None
+    if args.cp > 1:
+        if int(os.environ.get("WORLD_SIZE", "1")) == args.cp:
+            run_cp_ranks(args, w, aj)
+            return
+        if int(os.environ.get("WORLD_SIZE", "1")) != 1 or w.H % args.cp:
+            raise RuntimeError("--cp P runs with P ranks (--gpus P) or with one rank, and needs H to be a multiple of P")
+        # one rank: the per-rank call of a context-parallel group of P (H/P heads, whole sequence), no exchange
+        import dataclasses
+        w = dataclasses.replace(w, name=f"{w.name}/cp{args.cp}", H=w.H // args.cp)
+        cp_note = {"cp": args.cp, "cp_note": "per-rank kernel shape of a context-parallel group (H/P heads); "
+                                             "the all-to-all exchange is not part of this one-rank run"}
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -371,21 +493,32 @@ def main():
         peaks = measured_peaks()
         flops = w.executed_flops
         achieved = flops / (kernel_ms * 1e-3) / 1e12
-        traffic = None
-        if NCU_TRAFFIC_BYTES["bytes"] is not None:
-            wt = synth.WORKLOADS[NCU_TRAFFIC_BYTES["workload"]]
-            traffic = NCU_TRAFFIC_BYTES["bytes"] * algorithmic_bytes(w) / algorithmic_bytes(wt)
+        cap = NCU_TRAFFIC_BYTES[traffic_class(w)]
+        wt = synth.WORKLOADS[cap["workload"]]
+        traffic = cap["bytes"] * algorithmic_bytes(w) / algorithmic_bytes(wt)
+        # clock-normalised work: SM cycles one CTA spends per 64-key tile of a 128-row query tile (kernel time x
+        # sampled median SM clock x SMs / tiles), which separates the power state from the kernel's own cycles
+        tiles = w.B * w.H * ((w.Lq + 127) // 128) * ((w.Lk + 63) // 64)
+        sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+        cycles_per_tile = None
+        if clocks and clocks.get("sm_mhz"):
+            cycles_per_tile = kernel_ms * 1e-3 * clocks["sm_mhz"] * 1e6 * sm_count / tiles
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                     "frac": achieved / peaks["bf16_tflops"], "traffic": traffic,
                     "peak_source": f"{peaks['source']} burst cuBLAS bf16 (MEASURED_PEAKS.json)",
                     "kernel": "attn_jvp_fwd_kernel", "kernel_ms": kernel_ms, "flops_per_launch": flops,
                     "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"] if peaks["bf16_tflops_sustained"] else None,
                     "frac_of_datasheet": achieved / DATASHEET_BF16_TFLOPS,
-                    "algorithmic_bytes": algorithmic_bytes(w)}
+                    "algorithmic_bytes": algorithmic_bytes(w),
+                    "traffic_source": f"ncu capture on {cap['workload']} scaled by algorithmic bytes"
+                                      if cap["workload"] != w.name else f"ncu capture on {w.name}",
+                    "sm_cycles_per_key_tile": cycles_per_tile,
+                    "mma_cycles_per_key_tile_ideal": (w.executed_flops / (w.B * w.H * w.Lq * w.Lk * w.D)) * 128 * 64 * w.D / 8192.0}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": workload_config(w, extra={"splits": args.splits} if args.splits > 1 else None),
+                "config": workload_config(w, extra=dict(({"splits": args.splits} if args.splits > 1 else {}),
+                                                        **(cp_note or {}))),
                 "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * (2 if args.splits > 1 else 1),
                 "roofline": roofline,
                 "jvp_over_fwd": (kernel_ms / fwd_ms) if fwd_ms else None, "fwd_only_ms": fwd_ms,
