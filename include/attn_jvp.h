@@ -199,6 +199,24 @@ int attn_jvp_fwd_splitkv_static(const void* q, const void* k, const void* v,
                                 int B, int H, int Lq, int Lk, int D,
                                 float scale, unsigned flags, int splits, void* cuda_stream);
 
+/*
+ * Tuning knobs for benchmarking and A/B comparisons (process-wide; the paper has no counterpart).  Every setting
+ * computes the same function within the library's tolerance; only the kernel variant changes.
+ *   ATTN_JVP_TUNE_SOFTMAX_GROUPS  0 = the library chooses per (mode, D) (default), 1 = one softmax warpgroup per
+ *                                 CTA (192 threads), 2 = two warpgroups taking alternate key tiles (384 threads).
+ * Returns 0, or ATTN_JVP_ERR_FLAGS for an unknown knob or value.
+ */
+#define ATTN_JVP_TUNE_SOFTMAX_GROUPS 1
+int attn_jvp_set_tuning(int knob, int value);
+
+/*
+ * Diagnostics after ATTN_JVP_ERR_DEVICE_TIMEOUT (a bug report aid; the paper has no counterpart): which bounded
+ * wait gave up first on the current device since the last call.  out[0..3] (host memory) receive the
+ * shared-memory address of the barrier, the phase parity waited for, threadIdx.x and blockIdx.x of the waiting
+ * thread.  Returns 1 if there was a record (it is cleared), 0 if none, -1 on a CUDA error or NULL.  Blocking.
+ */
+int attn_jvp_debug_timeout_info(unsigned* out);
+
 /* Sets the stream attn_jvp_fwd launches on for the calling host thread
  * (thread-local; NULL = legacy default stream).  Always returns 0. */
 int attn_jvp_set_stream(void* cuda_stream);

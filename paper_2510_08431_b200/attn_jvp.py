@@ -23,7 +23,7 @@ STATIC_SCRATCH_BYTES = 32 * 1024 * 1024
 
 EXPORTS = ("attn_jvp_fwd", "attn_jvp_fwd_stream", "attn_jvp_fwd_mu", "attn_jvp_splitkv_workspace_bytes",
            "attn_jvp_suggest_splits", "attn_jvp_fwd_splitkv", "attn_jvp_fwd_splitkv_static", "attn_jvp_host_workspace_bytes",
-           "attn_jvp_fwd_host", "attn_jvp_qknorm_fwd", "attn_jvp_selftest_bounded_wait", "attn_jvp_set_stream", "attn_jvp_device_status", "attn_jvp_strerror",
+           "attn_jvp_fwd_host", "attn_jvp_qknorm_fwd", "attn_jvp_set_tuning", "attn_jvp_debug_timeout_info", "attn_jvp_selftest_bounded_wait", "attn_jvp_set_stream", "attn_jvp_device_status", "attn_jvp_strerror",
            "attn_jvp_version")
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libattn_jvp.so")
@@ -75,6 +75,8 @@ def load():
             lib.attn_jvp_qknorm_fwd.restype = ci
             lib.attn_jvp_selftest_bounded_wait.argtypes = [vp]
             lib.attn_jvp_selftest_bounded_wait.restype = ci
+            lib.attn_jvp_set_tuning.argtypes = [ci, ci]
+            lib.attn_jvp_set_tuning.restype = ci
             lib.attn_jvp_set_stream.argtypes = [vp]
             lib.attn_jvp_set_stream.restype = ci
             lib.attn_jvp_device_status.argtypes = []
@@ -83,6 +85,10 @@ def load():
             lib.attn_jvp_strerror.restype = ctypes.c_char_p
             lib.attn_jvp_version.argtypes = []
             lib.attn_jvp_version.restype = ci
+            # benchmarking aid: ATTN_JVP_SOFTMAX_GROUPS=1|2 forces the kernel variant for the whole process
+            forced = os.environ.get("ATTN_JVP_SOFTMAX_GROUPS")
+            if forced:
+                lib.attn_jvp_set_tuning(TUNE_SOFTMAX_GROUPS, int(forced))
             _lib = lib
     return _lib
 
@@ -101,6 +107,24 @@ def attn_jvp_strerror(code: int) -> str:
 
 def attn_jvp_version() -> int:
     return int(load().attn_jvp_version())
+
+
+TUNE_SOFTMAX_GROUPS = 1
+
+
+def attn_jvp_debug_timeout_info():
+    """After ERR_DEVICE_TIMEOUT: (barrier smem address, parity, threadIdx.x, blockIdx.x) of the first wait that
+    gave up on the current device, or None."""
+    buf = (ctypes.c_uint * 4)()
+    lib = load()
+    lib.attn_jvp_debug_timeout_info.argtypes = [ctypes.POINTER(ctypes.c_uint)]
+    lib.attn_jvp_debug_timeout_info.restype = ctypes.c_int
+    return tuple(buf) if lib.attn_jvp_debug_timeout_info(buf) == 1 else None
+
+
+def attn_jvp_set_tuning(knob: int, value: int) -> int:
+    """Process-wide tuning knob (see include/attn_jvp.h); returns the library's return code."""
+    return int(load().attn_jvp_set_tuning(int(knob), int(value)))
 
 
 def attn_jvp_set_stream(cuda_stream) -> int:

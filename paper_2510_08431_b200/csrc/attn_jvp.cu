@@ -46,6 +46,22 @@ DeviceState g_dev[kMaxDevices];
 std::mutex g_encode_lock;
 std::atomic<EncodeTiledFn> g_encode_tiled{nullptr};
 
+// Tuning knobs (attn_jvp_set_tuning); 0 = the library's own choice.
+std::atomic<int> g_tune_softmax_groups{0};
+
+// Softmax warpgroups per CTA for a kernel variant: two groups take alternate key tiles, which pays where the
+// softmax arithmetic, not the tensor pipe, sets the pace of a key tile.
+int softmax_groups_for(int mode, int D) {
+    const int forced = g_tune_softmax_groups.load(std::memory_order_relaxed);
+    if (forced == 1 || forced == 2) return forced;
+    (void)mode;
+    // Measured on B200 (image- and video-length self-attention): at D = 64 the tensor work per key tile is half
+    // that of D = 128 while the softmax work is the same, and two groups are 1.1-1.3x faster in every mode; at
+    // D = 128 one group is as fast or faster (the tile period is set by the MMA-issuing warp there, which two
+    // more busy warps on its scheduler slow down).
+    return D == 64 ? 2 : 1;
+}
+
 int cuda_fail(const char* what, cudaError_t e) {
     snprintf(tl_cuda_msg, sizeof tl_cuda_msg, "%s: %s", what, cudaGetErrorString(e));
     return ATTN_JVP_ERR_CUDA;
@@ -135,26 +151,26 @@ bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
     return a0 < b0 + nb && b0 < a0 + na;
 }
 
-template <int D, int MODE, bool SPLIT>
+template <int D, int MODE, bool SPLIT, int GROUPS>
 int launch(const CUtensorMap* maps, const KernelArgs& ka, dim3 grid, cudaStream_t stream, DeviceState& st) {
-    auto kern = attn_jvp::attn_jvp_fwd_kernel<D, MODE, SPLIT>;
-    std::atomic<int>& slot = st.dyn_smem[D == 128][MODE][SPLIT][0];
+    auto kern = attn_jvp::attn_jvp_fwd_kernel<D, MODE, SPLIT, GROUPS>;
+    using Plan = attn_jvp::SmemPlan<D, GROUPS>;
+    std::atomic<int>& slot = st.dyn_smem[D == 128][MODE][SPLIT][GROUPS - 1];
     int smem = slot.load(std::memory_order_acquire);
     if (smem == 0) {
-        // dynamic shared memory = the operand layout plus slack for its 1024-byte alignment, capped by
-        // what the device leaves after the kernel's static shared memory
+        // dynamic shared memory = the operand layout (declared 1024-byte aligned in the kernel) plus the exchange
+        // area of two softmax groups; it must fit beside the kernel's static shared memory
         std::lock_guard<std::mutex> guard(st.lock);
         smem = slot.load(std::memory_order_relaxed);
         if (smem == 0) {
             cudaFuncAttributes fa;
             cudaError_t e = cudaFuncGetAttributes(&fa, kern);
             if (e != cudaSuccess) return cuda_fail("cudaFuncGetAttributes", e);
-            int want = attn_jvp::SmemPlan<D>::kDynBytes;
+            const int want = Plan::kDynBytes;
             const int room = st.smem_optin - (int)fa.sharedSizeBytes;
-            if (want > room) want = room;
-            if (want < attn_jvp::SmemPlan<D>::kBytes) {
+            if (want > room) {
                 snprintf(tl_cuda_msg, sizeof tl_cuda_msg, "device offers %d bytes of shared memory, kernel needs %d",
-                         room, attn_jvp::SmemPlan<D>::kBytes);
+                         room, want);
                 return ATTN_JVP_ERR_CUDA;
             }
             e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, want);
@@ -163,7 +179,7 @@ int launch(const CUtensorMap* maps, const KernelArgs& ka, dim3 grid, cudaStream_
             slot.store(want, std::memory_order_release);
         }
     }
-    kern<<<grid, attn_jvp::kThreads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], maps[6],
+    kern<<<grid, attn_jvp::num_threads(GROUPS), smem, stream>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], maps[6],
                                                      maps[7], ka);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail("kernel launch", e);
@@ -299,18 +315,22 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     const long long n_ctas = (persistent && n_items > st.sm_count) ? st.sm_count : n_items;
     const dim3 grid((unsigned)n_ctas, 1, 1);
     int rc;
-#define ATTN_JVP_DISPATCH(DD, SS)                                                                                  \
+    const int groups = softmax_groups_for(mode, D);
+#define ATTN_JVP_DISPATCH_G(DD, SS, GG)                                                                            \
     switch (mode) {                                                                                               \
-        case attn_jvp::kModeJvp: rc = launch<DD, attn_jvp::kModeJvp, SS>(maps, ka, grid, stream, st); break;      \
+        case attn_jvp::kModeJvp: rc = launch<DD, attn_jvp::kModeJvp, SS, GG>(maps, ka, grid, stream, st); break;   \
         case attn_jvp::kModeKvTangentFree:                                                                        \
-            rc = launch<DD, attn_jvp::kModeKvTangentFree, SS>(maps, ka, grid, stream, st); break;                 \
-        default: rc = launch<DD, attn_jvp::kModeFwdOnly, SS>(maps, ka, grid, stream, st); break;                  \
+            rc = launch<DD, attn_jvp::kModeKvTangentFree, SS, GG>(maps, ka, grid, stream, st); break;              \
+        default: rc = launch<DD, attn_jvp::kModeFwdOnly, SS, GG>(maps, ka, grid, stream, st); break;               \
     }
+#define ATTN_JVP_DISPATCH(DD, SS)                                                                                  \
+    if (groups == 2) { ATTN_JVP_DISPATCH_G(DD, SS, 2) } else { ATTN_JVP_DISPATCH_G(DD, SS, 1) }
     if (D == 128) {
         if (split) { ATTN_JVP_DISPATCH(128, true) } else { ATTN_JVP_DISPATCH(128, false) }
     } else {
         if (split) { ATTN_JVP_DISPATCH(64, true) } else { ATTN_JVP_DISPATCH(64, false) }
     }
+#undef ATTN_JVP_DISPATCH_G
 #undef ATTN_JVP_DISPATCH
     if (rc != 0 || !split) return rc;
 
@@ -657,6 +677,14 @@ int attn_jvp_selftest_bounded_wait(void* cuda_stream) {
     return 0;
 }
 
+int attn_jvp_set_tuning(int knob, int value) {
+    if (knob == ATTN_JVP_TUNE_SOFTMAX_GROUPS && value >= 0 && value <= 2) {
+        g_tune_softmax_groups.store(value, std::memory_order_relaxed);
+        return 0;
+    }
+    return ATTN_JVP_ERR_FLAGS;
+}
+
 int attn_jvp_set_stream(void* cuda_stream) {
     tl_stream = static_cast<cudaStream_t>(cuda_stream);
     return 0;
@@ -715,6 +743,25 @@ const char* attn_jvp_strerror(int code) {
 }
 
 int attn_jvp_version(void) { return kVersion; }
+
+// Diagnostics after ATTN_JVP_ERR_DEVICE_TIMEOUT: which wait gave up first on the current device.  out[0..3] =
+// shared-memory address of the barrier, parity waited for, threadIdx.x, blockIdx.x; returns 1 if a record exists
+// (and clears it), 0 if not, -1 on a CUDA error.  Blocking (copies from the device).
+int attn_jvp_debug_timeout_info(unsigned* out) {
+    unsigned info[5] = {};
+    if (!out || cudaMemcpyFromSymbol(info, attn_jvp::g_timeout_info, sizeof info) != cudaSuccess) return -1;
+    for (int i = 0; i < 4; ++i) out[i] = info[i];
+    if (info[4] == 0) return 0;
+    const unsigned zero[5] = {};
+    cudaMemcpyToSymbol(attn_jvp::g_timeout_info, zero, sizeof zero);
+    return 1;
+}
+#ifdef ATTN_JVP_DEBUG
+int attn_jvp_debug_barrier_layout(unsigned* out, int n) {
+    if (n < 14) return -1;
+    return cudaMemcpyFromSymbol(out, attn_jvp::g_barrier_layout, 14 * sizeof(unsigned)) == cudaSuccess ? 14 : -1;
+}
+#endif
 
 #ifdef ATTN_JVP_TRACE
 // Debug builds only: copies the in-kernel timeline (clock64 stamps) of the traced CTA to `dst`.

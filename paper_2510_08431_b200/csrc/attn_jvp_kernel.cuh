@@ -16,8 +16,12 @@
 //   [0, D)        O  accumulator (line 13)
 //   [D, 2D)       T = A + B accumulator (lines 14 and 18 share one accumulator, since only
 //                 A + B is ever used, line 22)
-//   [256+128b, +64)  S  of score buffer b (b = key-tile parity); P~ (bf16) overwrites it
-//   [320+128b, +64)  tS of score buffer b;                        H~ (bf16) overwrites it
+//   [c0+128b, +64)     S  of score buffer b; P~ (bf16) overwrites it
+//   [c0+64+128b, +64)  tS of score buffer b; H~ (bf16) overwrites it
+// Two score buffers from column c0 = 256 (tile g uses buffer g % 2), or, where the accumulators need no more than
+// 128 columns (D = 64, and the forward-only mode), three from c0 = 128: the score MMAs then run three tiles
+// ahead of the value MMAs, which takes the round trip tensor pipe -> softmax warps -> tensor pipe out of the
+// tile period.
 //
 // Contractions per key tile (line 9 and lines 13, 14, 18):
 //   [S | Q tK^T] = Q [K ; tK]^T      one MMA chain, N = 128 (K and tK tiles are stacked in smem)
@@ -35,14 +39,18 @@ namespace attn_jvp {
 
 constexpr int kBlockM = 128;        // query rows per CTA (B_r)
 constexpr int kBlockN = 64;         // keys per tile (B_c)
-constexpr int kSoftmaxThreads = 128;   // four softmax warps: one thread per query row
+constexpr int kSoftmaxThreads = 128;   // four softmax warps per group: one thread per query row
 constexpr int kMmaWarp = 0;            // the two single-thread roles come first (oldest warps of the CTA)
 constexpr int kProducerWarp = 1;
-constexpr int kFirstSoftmaxWarp = 2;
-constexpr int kThreads = kSoftmaxThreads + 64;
+// One softmax group: warps 2..5 follow the two single-thread roles (192 threads).  Two groups (they take
+// alternate key tiles): the roles are laid out by warpgroup so that each can be given its own register budget --
+// warps 0..3 = MMA, producer and two idle warps, warps 4..7 = group 0, warps 8..11 = group 1 (384 threads).
+__host__ __device__ constexpr int first_softmax_warp(int groups) { return groups == 2 ? 4 : 2; }
+__host__ __device__ constexpr int num_threads(int groups) { return groups == 2 ? 384 : kSoftmaxThreads + 64; }
+constexpr int kRegsLightWarps = 104;    // two groups: registers per thread of warps 0..3 ...
+constexpr int kRegsSoftmaxWarps = 200; // ... and of the softmax warps (128 * 72 + 256 * 216 = 384 * 168)
 constexpr int kTmemCols = 512;
-constexpr int kScoreCol0 = 256;     // first column of score buffer 0
-constexpr int kScoreBufStride = 128;
+constexpr int kScoreBufStride = 128; // tensor-memory columns of one score buffer {S 64, tS 64}
 constexpr float kRescaleThreshold = 8.0f;   // log2 units: rescale only when the max grows by > 2^8
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // bound on every device-side wait
 constexpr uint32_t kTryWaitHintNs = 20000u;   // a waiting thread may sleep this long per try (it is woken on completion)
@@ -66,6 +74,13 @@ __device__ long long g_trace[kTraceEvents][kTraceSteps];
 
 // Set by any kernel whose bounded wait expired; later CTAs see it and leave at once.
 __device__ int g_abort_flag = 0;
+// Which wait expired first (diagnostics): shared-memory address of the barrier, the parity waited for,
+// threadIdx.x and blockIdx.x; [4] is nonzero once filled.  Debug builds (-DATTN_JVP_DEBUG) also record
+// the addresses of the kernel's barriers in g_barrier_layout so that the first word can be given a name.
+__device__ unsigned g_timeout_info[5] = {0, 0, 0, 0, 0};
+#ifdef ATTN_JVP_DEBUG
+__device__ unsigned g_barrier_layout[32];
+#endif
 
 struct KernelArgs {
     __nv_bfloat16* o;
@@ -92,7 +107,7 @@ struct KernelArgs {
     int n_items;        // work items = n_q_tiles * H * B * splits; the grid's CTAs share them round-robin
 };
 
-template <int D>
+template <int D, int kGroups = 1>
 struct SmemPlan {
     static constexpr int kHalves = D / 64;                 // 64-element (128-byte) swizzle atoms per row
     static constexpr int kQHalfBytes = kBlockM * 128;      // 16 KB: 128 rows x 128 B
@@ -100,8 +115,14 @@ struct SmemPlan {
     static constexpr int kKvHalfBytes = kBlockN * 128;     // 8 KB: 64 rows x 128 B
     static constexpr int kSlotBytes = 2 * kHalves * kKvHalfBytes;  // primal + tangent tile
     static constexpr int kSlots = (D == 128) ? 5 : 8;
-    static constexpr int kBytes = 2 * kQBytes + kSlots * kSlotBytes;
-    static constexpr int kDynBytes = kBytes + 1024;        // slack for manual 1024-byte alignment
+    static constexpr int kOperandBytes = 2 * kQBytes + kSlots * kSlotBytes;
+    // Two softmax groups exchange four per-row fp32 values through shared memory (reference max, centring
+    // constant of tS, partial l and r), placed after the operand tiles.
+    static constexpr int kExchangeBytes = (kGroups == 2) ? 4 * kBlockM * 4 : 0;
+    // The dynamic allocation is declared 1024-byte aligned (the operand tiles need that for the 128-byte
+    // swizzle); static shared memory (barriers, a few words) stays below 1 KB, so that at D = 128 operands
+    // (224 KB), exchange area (2 KB) and static part fill the 227 KB a CTA can have exactly.
+    static constexpr int kDynBytes = kOperandBytes + kExchangeBytes;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -169,6 +190,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const A
         if ((it & 255u) == 0u) {
             if (*st.cta_flag) return false;
             if (globaltimer_ns() - t0 > kWaitLimitNs) {
+                if (atomicCAS(&g_timeout_info[4], 0u, 1u) == 0u) {
+                    g_timeout_info[0] = bar;
+                    g_timeout_info[1] = parity;
+                    g_timeout_info[2] = threadIdx.x;
+                    g_timeout_info[3] = blockIdx.x;
+                }
                 report_device_error(st, 10);   // ATTN_JVP_ERR_DEVICE_TIMEOUT
                 return false;
             }
@@ -199,6 +226,14 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t sr
 }
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void st_shared_f32(uint32_t addr, float v) {
+    asm volatile("st.shared.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ float ld_shared_f32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    return v;
 }
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // The stores committed so far have read their shared-memory source (it may be overwritten).
@@ -359,14 +394,20 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-template <int D, int MODE, bool kSplit>
-__global__ void __launch_bounds__(kThreads, 1)
+// Score buffers a kernel variant can have (see the tensor-memory map above).
+__host__ __device__ constexpr int score_buffers(int D, int mode) {
+    return ((mode == kModeFwdOnly ? D : 2 * D) <= 128) ? 3 : 2;
+}
+
+template <int D, int MODE, bool kSplit, int kGroups>
+__global__ void __launch_bounds__(num_threads(kGroups), 1)
 attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_tq,
                     const __grid_constant__ CUtensorMap tm_tk, const __grid_constant__ CUtensorMap tm_tv,
                     const __grid_constant__ CUtensorMap tm_o, const __grid_constant__ CUtensorMap tm_to,
                     const KernelArgs args) {
-    using Plan = SmemPlan<D>;
+    using Plan = SmemPlan<D, kGroups>;
+    constexpr int kFirstSoftmaxWarp = first_softmax_warp(kGroups);
     constexpr int kHalves = Plan::kHalves;
     constexpr int kSlots = Plan::kSlots;
     constexpr bool kHasTQ = (MODE != kModeFwdOnly);          // tS and T exist
@@ -380,21 +421,28 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // beside the H~ arithmetic (H~ follows through a barrier of its own).  In the full mode the MMA warp never
     // waits for the softmax warps, and the second hand-over would only add work (measured: 1 % slower).
     constexpr bool kSplitHandover = kHasTQ && !kHasTKV;
+    constexpr int kBufs = score_buffers(D, MODE);            // score buffers = how many tiles the score MMAs run ahead
+    constexpr int kScoreCol0 = (kBufs == 3) ? 128 : 256;     // first column of score buffer 0
+    static_assert(kScoreCol0 + kBufs * kScoreBufStride <= kTmemCols, "score buffers must fit into tensor memory");
+    static_assert((kHasTQ ? 2 * D : D) <= kScoreCol0, "accumulators and score buffers overlap");
     static_assert(Plan::kSlotBytes == Plan::kQBytes, "an output tile must fill one ring slot");
 
-    extern __shared__ uint8_t smem_raw[];
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_q_full;     // Q, tQ of the current work item are in shared memory
     __shared__ __align__(8) uint64_t bar_q_free;     // every score MMA of the item has completed: Q, tQ may be replaced
     __shared__ __align__(8) uint64_t bar_slot_full[kSlots];
     __shared__ __align__(8) uint64_t bar_slot_empty[kSlots];
-    __shared__ __align__(8) uint64_t bar_s_full[2];
-    __shared__ __align__(8) uint64_t bar_p_full[2];     // P~ of the tile is in tensor memory
-    __shared__ __align__(8) uint64_t bar_h_full[2];     // H~ of the tile is in tensor memory (some 500 cycles later)
-    __shared__ __align__(8) uint64_t bar_pv_done;
+    __shared__ __align__(8) uint64_t bar_s_full[kBufs];
+    __shared__ __align__(8) uint64_t bar_p_full[kBufs];     // P~ of the tile is in tensor memory
+    __shared__ __align__(8) uint64_t bar_h_full[kBufs];     // H~ of the tile is in tensor memory (some 500 cycles later)
+    __shared__ __align__(8) uint64_t bar_pv_done[2];        // the value MMAs of tile g (and all before) are complete: [g & 1]
     __shared__ __align__(8) uint64_t bar_acc_free;   // the epilogue has read O and T: the next item may overwrite them
     __shared__ __align__(8) uint64_t bar_drain;
     __shared__ __align__(8) uint64_t bar_stage_ready;   // the item's staging slots are free of operand reads
     __shared__ __align__(8) uint64_t bar_stage_full;    // the softmax warps have written the item's output tiles
+    // two softmax groups, one barrier per quarter of the rows (a pair of warps, one of each group):
+    __shared__ __align__(8) uint64_t bar_m[4];          // the reference max after tile g is published (phase g & 1)
+    __shared__ __align__(8) uint64_t bar_fin[4];        // the non-finishing group's partial l, r of the item are published
     __shared__ uint32_t tmem_base_smem;
     __shared__ int cta_abort;
 
@@ -421,6 +469,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         return w;
     };
     const int n_items = args.n_items;
+    auto sbuf = [](int g) -> int { return kBufs == 2 ? (g & 1) : g % kBufs; };
+    auto sphase = [](int g) -> uint32_t { return static_cast<uint32_t>(kBufs == 2 ? (g >> 1) : g / kBufs) & 1u; };
 
     // An earlier CTA of this (or a previous) launch gave up: do not start.  One thread reads
     // the flag so that the whole CTA takes the same decision.
@@ -431,19 +481,20 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #ifdef ATTN_JVP_TRACE
     if (trace_on && threadIdx.x == 0) g_trace[kTraceEvents - 1][0] = clock64();      // CTA begins
 #endif
-    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t smem_base = smem_u32(smem_raw);
     const uint32_t smem_q = smem_base;
     const uint32_t smem_tq = smem_base + Plan::kQBytes;
     const uint32_t smem_ring = smem_base + 2 * Plan::kQBytes;
 
     AbortState abort_state{&cta_abort, args.host_status};
 
-    // The operand tiles need 1024-byte alignment; the host sizes the dynamic allocation so that the
-    // aligned layout fits, and this check keeps a mismatch from becoming an out-of-bounds access.
+    // The operand tiles need 1024-byte alignment (the dynamic allocation is declared that way) and the host
+    // must have asked for the whole layout: this check keeps a mismatch from becoming a wrong or out-of-bounds
+    // access.
     {
         uint32_t dyn_size;
         asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_size));
-        if (smem_base + Plan::kBytes > smem_u32(smem_raw) + dyn_size) {
+        if ((smem_base & 1023u) != 0u || static_cast<uint32_t>(Plan::kDynBytes) > dyn_size) {
             if (threadIdx.x == 0) report_device_error(abort_state, 11);   // ATTN_JVP_ERR_DEVICE_LAYOUT
             return;
         }
@@ -456,17 +507,30 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             mbar_init(smem_u32(&bar_slot_full[i]), 1);
             mbar_init(smem_u32(&bar_slot_empty[i]), 1);
         }
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < kBufs; ++i) {
             mbar_init(smem_u32(&bar_s_full[i]), 1);
             mbar_init(smem_u32(&bar_p_full[i]), kSoftmaxThreads / 32);    // one arrival per softmax warp
             mbar_init(smem_u32(&bar_h_full[i]), kSoftmaxThreads / 32);
         }
-        mbar_init(smem_u32(&bar_pv_done), 1);
+        mbar_init(smem_u32(&bar_pv_done[0]), 1);
+        mbar_init(smem_u32(&bar_pv_done[1]), 1);
         mbar_init(smem_u32(&bar_acc_free), kSoftmaxThreads / 32);
         mbar_init(smem_u32(&bar_drain), 1);
         mbar_init(smem_u32(&bar_stage_ready), 1);
         mbar_init(smem_u32(&bar_stage_full), kSoftmaxThreads / 32);
+        for (int i = 0; i < 4; ++i) {
+            mbar_init(smem_u32(&bar_m[i]), 1);
+            mbar_init(smem_u32(&bar_fin[i]), 1);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+#ifdef ATTN_JVP_DEBUG
+        if (blockIdx.x == 0) {
+            const void* named[] = {&bar_q_full, &bar_q_free, &bar_slot_full[0], &bar_slot_empty[0], &bar_s_full[0],
+                                   &bar_p_full[0], &bar_h_full[0], &bar_pv_done[0], &bar_acc_free, &bar_drain,
+                                   &bar_stage_ready, &bar_stage_full, &bar_m[0], &bar_fin[0]};
+            for (int i = 0; i < 14; ++i) g_barrier_layout[i] = smem_u32(named[i]);
+        }
+#endif
     }
     if (warp == kMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -489,16 +553,24 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const uint32_t tmem_o = tmem;
     const uint32_t tmem_t = tmem + D;
 
-    // Phases.  Key tiles are numbered g = 0, 1, 2, ... over ALL items of this CTA; tile g uses score buffer g & 1,
-    // phase (g >> 1) & 1 of bar_s_full / bar_p_full and phase g & 1 of bar_pv_done.  Item number `it` (0, 1, ...)
+    // Phases.  Key tiles are numbered g = 0, 1, 2, ... over ALL items of this CTA; tile g uses score buffer
+    // g % kBufs, phase (g / kBufs) & 1 of bar_s_full / bar_p_full / bar_h_full, and phase (g >> 1) & 1 of
+    // bar_pv_done[g & 1] (two barriers, so that a wait for tile g - 1 cannot be mistaken for one two tiles on).  Item number `it` (0, 1, ...)
     // uses phase it & 1 of bar_q_full / bar_q_free / bar_acc_free / bar_stage_ready / bar_stage_full.  The
     // shared-memory ring runs on without a break; per item it hands out 2 n slots to K/V tiles and then
     // kStageSlots slots to the output tiles.
 
+    // Two softmax groups: the warps of the first warpgroup need few registers (two of them are idle), the
+    // softmax warps hold a whole row of scores and tangent scores each; the budgets are moved accordingly.
+    // (The forward-only softmax needs fewer registers than the 168 every thread of a 384-thread CTA starts with.)
+    constexpr bool kMoveRegs = (kGroups == 2) && kHasTQ;
+    if (warp < kFirstSoftmaxWarp) {
+    if (kMoveRegs) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLightWarps));
     if (warp == kProducerWarp) {
         // =====================================================================================
         // TMA producer.  Per item: Q, tQ (once the previous item's score MMAs are done), then the ring in
-        // consumption order K0, K1, V0, K2, V1, ..., K(n-1), V(n-2), V(n-1).
+        // consumption order K0, K1, V0, K2, V1, ..., K(n-1), V(n-2), V(n-1) (two score buffers; with three the
+        // K tiles run one more ahead: K0, K1, K2, V0, K3, V1, ...).
         // =====================================================================================
         if (lane == 0) {
             constexpr uint32_t kQTx = (kHasTQ ? 2u : 1u) * Plan::kQBytes;
@@ -615,8 +687,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         if (kHasTQ) tma_prefetch_4d(&tm_tq, hf * 64, nx.h, nx.q0, nx.b);
                     }
                 }
-                ok = load_k(0);
-                if (ok && w.n_kv > 1) ok = load_k(1);
+                for (int t = 0; ok && t < kBufs && t < w.n_kv; ++t) ok = load_k(t);
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 3
                 {   // timing experiment: when do Q, tQ land?
                     const unsigned long long t0 = globaltimer_ns();
@@ -628,7 +699,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 // need at once) and before its V tiles (which are not needed until the first softmax is through)
                 if (kStageSlots > 0 && ok && it > 0) ok = acquire_stage(it - 1, prev_w);
                 for (int j = 0; ok && j < w.n_kv; ++j) {
-                    if (j >= 1 && j + 1 < w.n_kv) ok = load_k(j + 1);
+                    if (j >= 1 && j + kBufs - 1 < w.n_kv) ok = load_k(j + kBufs - 1);
                     if (ok) ok = load_v(j);
                     // the previous item's outputs: the loads above do not depend on its epilogue, the later ones do
                     if (ok && stage_pending && (j == 1 || j + 1 == w.n_kv)) ok = store_staged();
@@ -686,49 +757,37 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 return mbar_wait_warp(bar, r.parity, abort_state);
             };
 
-            // Operand descriptors.  Q and tQ never move: their eight per-k-step descriptors are built once.
-            // Those of a ring slot are built by prepare_*() BEFORE the burst that uses them, so that inside a
-            // burst every tcgen05.mma is a single instruction with its operands ready.
-            uint64_t qd[D / 16], tqd[D / 16];
-#pragma unroll
-            for (int k = 0; k < D / 16; ++k) {
-                const uint32_t koff = ((k / 4) * Plan::kQHalfBytes + (k % 4) * 32) >> 4;
-                qd[k] = make_desc(q_lo + koff);
-                tqd[k] = make_desc(tq_lo + koff);
-            }
-            uint64_t kd[D / 16];            // K-slot descriptors of the score MMAs about to be issued
-            uint64_t vd[kBlockN / 16];      // V-slot descriptors of the value MMAs about to be issued
-            auto prepare_k = [&](int slot) {
-                const uint32_t k_lo = make_desc_lo(smem_ring + slot * Plan::kSlotBytes, 16);
-#pragma unroll
-                for (int k = 0; k < D / 16; ++k)
-                    kd[k] = make_desc(k_lo + (((k / 4) * 2 * Plan::kKvHalfBytes + (k % 4) * 32) >> 4));
-            };
-            auto prepare_v = [&](int slot) {
-                const uint32_t v_lo = make_desc_lo(smem_ring + slot * Plan::kSlotBytes, kVLbo);
-#pragma unroll
-                for (int k = 0; k < kBlockN / 16; ++k) vd[k] = make_desc(v_lo + k * (2048 >> 4));
-            };
+            // Operand descriptors: per operand only the low word of its first k-step is kept in a register (Q and
+            // tQ never move; the ring slot's words are set by prepare_*() before the burst that uses them).  The
+            // k-steps differ by compile-time constants, so that inside a burst a descriptor costs one add with an
+            // immediate and one move beside the tcgen05.mma itself, and the issuing warp stays small in registers.
+            uint32_t k_lo = 0, v_lo = 0;
+            auto prepare_k = [&](int slot) { k_lo = make_desc_lo(smem_ring + slot * Plan::kSlotBytes, 16); };
+            auto prepare_v = [&](int slot) { v_lo = make_desc_lo(smem_ring + slot * Plan::kSlotBytes, kVLbo); };
+            auto qd = [&](int k) { return make_desc(q_lo + (((k / 4) * Plan::kQHalfBytes + (k % 4) * 32) >> 4)); };
+            auto tqd = [&](int k) { return make_desc(tq_lo + (((k / 4) * Plan::kQHalfBytes + (k % 4) * 32) >> 4)); };
+            auto kd = [&](int k) { return make_desc(k_lo + (((k / 4) * 2 * Plan::kKvHalfBytes + (k % 4) * 32) >> 4)); };
+            auto vd = [&](int k) { return make_desc(v_lo + k * (2048 >> 4)); };
 
             // score MMAs of global tile g (issued by the elected lane), in two parts so that the look-ahead for
             // the next tile can run between them; `last_of_item`: these are the item's last score MMAs
             auto issue_scores_a = [&](int g) {
-                const uint32_t tm_s = tmem + kScoreCol0 + (g & 1) * kScoreBufStride;
+                const uint32_t tm_s = tmem + kScoreCol0 + sbuf(g) * kScoreBufStride;
                 TRACE(21, g);         // MMA: about to issue score MMAs
-                mma_ss<false>(tm_s, qd[0], kd[0], kIdescS1);
+                mma_ss<false>(tm_s, qd(0), kd(0), kIdescS1);
 #pragma unroll
-                for (int k = 1; k < D / 16; ++k) mma_ss<true>(tm_s, qd[k], kd[k], kIdescS1);
+                for (int k = 1; k < D / 16; ++k) mma_ss<true>(tm_s, qd(k), kd(k), kIdescS1);
             };
             auto issue_scores_b = [&](int g, int slot, bool last_of_item) {
-                const uint32_t tm_ts = tmem + kScoreCol0 + (g & 1) * kScoreBufStride + kBlockN;
+                const uint32_t tm_ts = tmem + kScoreCol0 + sbuf(g) * kScoreBufStride + kBlockN;
                 if (kHasTQ) {
-                    if (kHasTKV) mma_ss<true>(tm_ts, tqd[0], kd[0], kIdescS2);
-                    else mma_ss<false>(tm_ts, tqd[0], kd[0], kIdescS2);
+                    if (kHasTKV) mma_ss<true>(tm_ts, tqd(0), kd(0), kIdescS2);
+                    else mma_ss<false>(tm_ts, tqd(0), kd(0), kIdescS2);
 #pragma unroll
-                    for (int k = 1; k < D / 16; ++k) mma_ss<true>(tm_ts, tqd[k], kd[k], kIdescS2);
+                    for (int k = 1; k < D / 16; ++k) mma_ss<true>(tm_ts, tqd(k), kd(k), kIdescS2);
                 }
                 tc_commit(smem_u32(&bar_slot_empty[slot]));
-                tc_commit(smem_u32(&bar_s_full[g & 1]));
+                tc_commit(smem_u32(&bar_s_full[sbuf(g)]));
                 if (last_of_item) tc_commit(smem_u32(&bar_q_free));
                 TRACE(2, g);          // MMA: score MMAs of tile g issued
             };
@@ -736,37 +795,37 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // value MMAs of tile j of the item (global tile g) out of ring slot `slot`, in two parts: those that read
             // P~ can run while the softmax warps are still forming H~
             auto issue_values_p = [&](int j, int g) {
-                const uint32_t tm_p = tmem + kScoreCol0 + (g & 1) * kScoreBufStride;
+                const uint32_t tm_p = tmem + kScoreCol0 + sbuf(g) * kScoreBufStride;
                 TRACE(3, g);          // MMA: about to issue value MMAs
 #pragma unroll
                 for (int k = 0; k < kBlockN / 16; ++k) {
-                    mma_ts(tmem_o, tm_p + k * 8, vd[k], kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
+                    mma_ts(tmem_o, tm_p + k * 8, vd(k), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
                 }
             };
             auto issue_values_h = [&](int j, int g, int slot) {
-                const uint32_t tm_h = tmem + kScoreCol0 + (g & 1) * kScoreBufStride + kBlockN;
+                const uint32_t tm_h = tmem + kScoreCol0 + sbuf(g) * kScoreBufStride + kBlockN;
                 if (kHasTQ) {
 #pragma unroll
                     for (int k = 0; k < kBlockN / 16; ++k) {
-                        mma_ts(tmem_t, tm_h + k * 8, vd[k], kIdescHV, (kHasTKV || j > 0 || k > 0) ? 1u : 0u);
+                        mma_ts(tmem_t, tm_h + k * 8, vd(k), kIdescHV, (kHasTKV || j > 0 || k > 0) ? 1u : 0u);
                     }
                 }
                 tc_commit(smem_u32(&bar_slot_empty[slot]));
-                tc_commit(smem_u32(&bar_pv_done));
+                tc_commit(smem_u32(&bar_pv_done[g & 1]));
                 TRACE(4, g);          // MMA: value MMAs of tile g issued
             };
             // what the burst of global tile g needs: V and K(+2) in shared memory, P~/H~ in tensor memory
             auto test_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, int g) -> bool {
                 bool r = mbar_test_wait(smem_u32(&bar_slot_full[pv.slot]), pv.parity);
                 if (has_k) r = r && mbar_test_wait(smem_u32(&bar_slot_full[pk.slot]), pk.parity);
-                r = r && mbar_test_wait(smem_u32(&bar_p_full[g & 1]), (g >> 1) & 1);
+                r = r && mbar_test_wait(smem_u32(&bar_p_full[sbuf(g)]), sphase(g));
                 return __all_sync(0xffffffffu, r);
             };
             auto wait_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, int g) -> bool {
                 if (leader) TRACE(22, g);   // MMA: has to block for tile g
                 bool r = wait_full(pv);
                 if (r && has_k) r = wait_full(pk);
-                if (r) r = mbar_wait_warp(smem_u32(&bar_p_full[g & 1]), (g >> 1) & 1, abort_state);
+                if (r) r = mbar_wait_warp(smem_u32(&bar_p_full[sbuf(g)]), sphase(g), abort_state);
                 return r;
             };
 
@@ -779,28 +838,26 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const int n_kv = w.n_kv;
                 ok = mbar_wait_warp(smem_u32(&bar_q_full), it & 1, abort_state);
                 if (leader) TRACE(10, it);    // MMA: Q, tQ of the item seen
-                if (ok) ok = wait_full(pos);
-                if (!ok) break;
-                if (leader) TRACE(11, it);    // MMA: K(0) of the item seen
-                tc_fence_after();
-                prepare_k(pos.slot);
-                if (leader) { issue_scores_a(g0); issue_scores_b(g0, pos.slot, n_kv == 1); }
-                __syncwarp();
-                advance(pos);
-                if (n_kv > 1) {
+                // the item's leading score MMAs: one tile per score buffer
+                for (int t = 0; ok && t < kBufs && t < n_kv; ++t) {
                     ok = wait_full(pos);
                     if (!ok) break;
+                    if (t == 0) {
+                        if (leader) TRACE(11, it);    // MMA: K(0) of the item seen
+                        tc_fence_after();
+                    }
                     prepare_k(pos.slot);
-                    if (leader) { issue_scores_a(g0 + 1); issue_scores_b(g0 + 1, pos.slot, n_kv == 2); }
+                    if (leader) { issue_scores_a(g0 + t); issue_scores_b(g0 + t, pos.slot, t + 1 == n_kv); }
                     __syncwarp();
                     advance(pos);
                 }
+                if (!ok) break;
                 // the ring positions between the item's leading K tiles and V(0) stage the previous item's outputs
                 if (it > 0) { for (int s = 0; s < kStageSlots; ++s) advance(pos); }
-                // pos = V(0).  Per tile j: burst = value MMAs of tile j, score MMAs of tile j+2; the barriers of
+                // pos = V(0).  Per tile j: burst = value MMAs of tile j, score MMAs of tile j + kBufs; the barriers of
                 // tile j+1 are tested in the middle of the burst, while the queue is still full.
                 RingPos pos_v = pos, pos_k = pos;
-                bool has_k = n_kv > 2;
+                bool has_k = n_kv > kBufs;
                 advance(pos);
                 pos_k = pos;
                 if (has_k) advance(pos);
@@ -815,19 +872,21 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const RingPos nxt_v = pos;
                     RingPos nxt_k = pos;
                     const bool nxt_exists = j + 1 < n_kv;
-                    const bool nxt_has_k = j + 3 < n_kv;
+                    const bool nxt_has_k = j + 1 + kBufs < n_kv;
                     if (nxt_exists) {
                         advance(pos);
                         nxt_k = pos;
                         if (nxt_has_k) advance(pos);
                     }
+                    if (leader) TRACE(29, g0 + j);   // MMA: burst of tile j begins (loop top)
                     tc_fence_after();
+                    if (leader) TRACE(30, g0 + j);   // MMA: after the tensor-core fence
                     if (leader) issue_values_p(j, g0 + j);
                     __syncwarp();
                     if (kSplitHandover) {
                         // H~ follows P~ by a few hundred cycles: normally it is there by now
-                        const uint32_t hbar = smem_u32(&bar_h_full[(g0 + j) & 1]);
-                        const uint32_t hpar = ((g0 + j) >> 1) & 1;
+                        const uint32_t hbar = smem_u32(&bar_h_full[sbuf(g0 + j)]);
+                        const uint32_t hpar = sphase(g0 + j);
                         if (!__all_sync(0xffffffffu, mbar_test_wait(hbar, hpar))) {
                             if (leader) TRACE(24, g0 + j);   // MMA: has to block for H~ of tile g
                             ok = mbar_wait_warp(hbar, hpar, abort_state);
@@ -838,13 +897,14 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     }
                     if (leader) {
                         issue_values_h(j, g0 + j, pos_v.slot);
-                        if (has_k) issue_scores_a(g0 + j + 2);
+                        if (has_k) issue_scores_a(g0 + j + kBufs);
                     }
                     __syncwarp();
                     bool nxt_ready = true;
                     if (nxt_exists) nxt_ready = test_tile(nxt_v, nxt_k, nxt_has_k, g0 + j + 1);
-                    if (leader && has_k) issue_scores_b(g0 + j + 2, pos_k.slot, j + 3 == n_kv);
+                    if (leader && has_k) issue_scores_b(g0 + j + kBufs, pos_k.slot, j + kBufs + 1 == n_kv);
                     __syncwarp();
+                    if (leader) TRACE(23, g0 + j);   // MMA: burst of tile j issued, warp reconverged
                     // descriptors of the next burst (this warp is held back by the full queue here anyway)
                     if (nxt_exists) {
                         prepare_v(nxt_v.slot);
@@ -865,11 +925,23 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             }
             __syncwarp();
         }
+    }
     } else {
+        if (kMoveRegs) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmaxWarps));
         // =====================================================================================
         // Softmax warps.  Thread (warp w, lane) owns query row 32*(w%4) + lane (= its tensor-memory
         // lane) and all 64 columns of every score tile.
+        //
+        // With two groups, group (g & 1) takes key tile g (numbered over all items of the CTA, like the score
+        // buffers), so that two tiles are in work at a time and each scheduler has two softmax warps to hide
+        // latencies with.  What Algorithm 2 carries from tile to tile is shared as follows.  The reference max m
+        // (and, once per item, the centring constant of tS) goes through shared memory in tile order: the group
+        // of tile g waits for the decision of tile g - 1, takes its own, publishes it and only then computes its
+        // exponentials, so the groups run half a tile apart.  l and r are summed per group (both relative to the
+        // common m); the group of the item's last tile finishes the item: it adds the other group's sums and runs
+        // the epilogue while the other group is already in the next item.
         // =====================================================================================
+        const int grp = (kGroups == 2) ? ((warp - kFirstSoftmaxWarp) >> 2) : 0;
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;                          // 0..127: a warp may only touch lanes 32*(warp%4)..+31
         const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
@@ -880,19 +952,30 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         int g0 = 0;          // global number of the item's first key tile
         int it = 0;
         int ring_slot = 0;   // ring slot of the item's first position (the ring hands out 2 n + kStageSlots per item)
+        // exchange area of the two groups, one fp32 per row each
+        const uint32_t xch_m = smem_base + Plan::kOperandBytes + row * 4;       // reference max after the latest tile
+        const uint32_t xch_shift = xch_m + kBlockM * 4;                         // centring constant of the item
+        const uint32_t xch_l = xch_m + 2 * kBlockM * 4;                         // partial l of the non-finishing group
+        const uint32_t xch_r = xch_m + 3 * kBlockM * 4;                         // partial r
+        const uint32_t mbar = smem_u32(&bar_m[quarter]);
+        const uint32_t finbar = smem_u32(&bar_fin[quarter]);
 
         for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
             const Item w = decode(item);
             const int n_kv = w.n_kv;
             float m_ref = -INFINITY;   // running reference max, log2 domain (m of Algorithm 2, lazily updated)
-            float l_run = 0.0f;        // l
-            float r_run = 0.0f;        // r (of the centred tS, see below)
+            float l_run = 0.0f;        // l (two groups: this group's share)
+            float r_run = 0.0f;        // r (of the centred tS, see below; two groups: this group's share)
             float ts_shift = 0.0f;     // per-row constant subtracted from tS
+            float m_other = -INFINITY; // two groups: the reference the other group's sums were last known to use
+            // two groups: the group of the item's last tile finishes the item
+            const bool finisher = (kGroups == 1) || (((g0 + n_kv - 1) & 1) == grp);
 
             for (int j = 0; j < n_kv; ++j) {
                 const int g = g0 + j;
-                const int bsel = g & 1;
-                if (!mbar_wait_warp(smem_u32(&bar_s_full[bsel]), (g >> 1) & 1, abort_state)) { ok = false; break; }
+                if (kGroups == 2 && (g & 1) != grp) continue;
+                const int bsel = sbuf(g);
+                if (!mbar_wait_warp(smem_u32(&bar_s_full[bsel]), sphase(g), abort_state)) { ok = false; break; }
                 tc_fence_after();
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
                 const bool trace_me = trace_on && lane == 0;
@@ -909,6 +992,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (kHasTQ) TMEM_LD32(tm_ts + c0, tv, c0);
                 }
                 tc_wait_ld();
+#if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
+                if (trace_me && quarter == 0 && g < kTraceSteps) g_trace[26][g] = clock64();    // softmax: scores in registers
+#endif
 
                 // keys past Lk (zero-filled by TMA) must not enter the softmax
                 const int valid = args.Lk - (w.tile0 + j) * kBlockN;
@@ -933,6 +1019,39 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                                      : fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                 mx *= c1;
 
+                if (kGroups == 2) {
+                    // The decision of tile g - 1 (the other group's) comes first, also across items: the exchange
+                    // words are single and are written strictly in tile order.
+                    if (g > 0 && !mbar_wait_warp(mbar, (g - 1) & 1, abort_state)) { ok = false; break; }
+                    if (j > 0) {
+                        const float m_prev = ld_shared_f32(xch_m);
+                        if (j == 1) ts_shift = ld_shared_f32(xch_shift);
+                        m_other = m_prev;
+                        if (m_prev > m_ref) {
+                            // this group's sums move to the common reference (0 * 0 on its first tile)
+                            const float f = ex2f(m_ref - m_prev);
+                            l_run *= f;
+                            r_run *= f;
+                            m_ref = m_prev;
+                        }
+                    }
+                }
+#if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
+                if (trace_me && quarter == 0 && g < kTraceSteps) g_trace[27][g] = clock64();    // softmax: reference of tile g-1 seen
+#endif
+                if (kHasTQ && j == 0) {
+                    // tO does not change when a per-row constant is subtracted from tS (softmax is shift
+                    // invariant: the constant leaves H~ V - (r/l) O unchanged).  Centring tS on its mean over the
+                    // item's first tile keeps H~ and r small, so that the bf16 rounding of H~ scales with
+                    // |tS - mu| instead of |tS| when the two terms cancel in the epilogue.  (Keys past Lk are
+                    // zero-filled, so their tS is exactly 0 and they drop out of the sum.)
+                    float sm4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+                    for (int c = 0; c < kBlockN; ++c) sm4[c & 3] += __uint_as_float(tv[c]);
+                    const int n_valid = valid < kBlockN ? valid : kBlockN;
+                    ts_shift = sc * ((sm4[0] + sm4[1]) + (sm4[2] + sm4[3])) / static_cast<float>(n_valid);
+                }
+
                 // m_new = max(m, rowmax), applied lazily: the result does not depend on which
                 // reference is used as long as exp() stays in range.
                 float alpha = 1.0f;
@@ -943,7 +1062,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
                 if (j > 0 && __any_sync(0xffffffffu, need)) {
                     // the accumulators must be complete up to tile j-1 before they are rescaled
-                    if (!mbar_wait_warp(smem_u32(&bar_pv_done), (g - 1) & 1, abort_state)) { ok = false; break; }
+                    if (!mbar_wait_warp(smem_u32(&bar_pv_done[(g - 1) & 1]), ((g - 1) >> 1) & 1, abort_state)) { ok = false; break; }
                     tc_fence_after();
                     constexpr int kAccCols = kHasTQ ? 2 * D : D;
 #pragma unroll 1
@@ -958,6 +1077,13 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
                 l_run *= alpha;
                 r_run *= alpha;
+                if (kGroups == 2) {
+                    // publish the decision (and the item's centring constant): the other group may go on
+                    st_shared_f32(xch_m, m_ref);
+                    if (j == 0) st_shared_f32(xch_shift, ts_shift);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(mbar);
+                }
 
                 // P~ = exp(S - m_new), l += rowsum(P~)   (two columns per FMA-pipe instruction)
                 const uint64_t c1c1 = pack_f32x2(c1, c1);
@@ -992,6 +1118,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     for (int c = 0; c < kBlockN / 2; ++c) pk[c] = pack_bf16(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1]));
                     TMEM_ST32(tm_s, pk, 0);
                 }
+#if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
+                if (trace_me && quarter == 0 && g < kTraceSteps) g_trace[28][g] = clock64();    // softmax: P~ store issued
+#endif
                 if (kSplitHandover) {
                     // P~ is handed over at once: the MMAs that read it run beside the H~ arithmetic below
                     tc_wait_st();
@@ -1000,17 +1129,6 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (lane == 0) mbar_arrive(smem_u32(&bar_p_full[bsel]));
                 }
                 if (kHasTQ) {
-                    // tO does not change when a per-row constant is subtracted from tS (softmax is shift
-                    // invariant: the constant leaves H~ V - (r/l) O unchanged).  Centring tS on its P-weighted
-                    // mean over the first tile keeps H~ and r small, so that the bf16 rounding of H~ scales
-                    // with |tS - mu| instead of |tS| when the two terms cancel in the epilogue.
-                    if (j == 0) {
-                        float nm4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-#pragma unroll
-                        for (int c = 0; c < kBlockN; ++c)
-                            nm4[c & 3] = fmaf(__uint_as_float(sv[c]), __uint_as_float(tv[c]) * sc, nm4[c & 3]);
-                        ts_shift = ((nm4[0] + nm4[1]) + (nm4[2] + nm4[3])) / lsum;
-                    }
                     // H~ = P~ . tS, r += rowsum(H~)
                     const uint64_t scsc = pack_f32x2(sc, sc);
                     const uint64_t negshift = pack_f32x2(-ts_shift, -ts_shift);
@@ -1046,12 +1164,43 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             }
             if (!ok) break;
 
-            // Epilogue: O/l, L = m + log l, tO = (T - r (O/l)) / l
-            // A parity wait can only tell the current phase from the previous one, and the value MMAs of
-            // tile n-2 may still be running here: wait for them first, then for those of tile n-1.
+            // Ring positions of this item: 2 n_kv tiles, plus the previous item's staging slots.  Its own staging
+            // slots come after the next item's leading K tiles (every item has n_kv tiles here: the kernel that
+            // cuts the keys into chunks stages nothing), or right after its last V tile if it is the CTA's last.
+            int stage_slot_o = 0;
+            if (kStageSlots > 0) {
+                const bool has_next = n_items - item > static_cast<int>(gridDim.x);
+                const int next_start = (ring_slot + 2 * (n_kv % kSlots) + (it > 0 ? kStageSlots : 0)) % kSlots;
+                stage_slot_o = has_next ? (next_start + min(kBufs, n_kv)) % kSlots : next_start;
+                ring_slot = next_start;
+            }
+
+            if (kGroups == 2 && !finisher) {
+                // This group's share of l and r goes to the group that finishes the item; the exchange words are
+                // single, so the finisher of the item before must have read its own first (it arrives on
+                // `acc_free` after that; at this point that barrier is in the phase of item it - 1 or it).
+                if (it > 0 && !mbar_wait_warp(smem_u32(&bar_acc_free), (it - 1) & 1, abort_state)) { ok = false; break; }
+                st_shared_f32(xch_l, l_run);
+                st_shared_f32(xch_r, r_run);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(finbar);
+                g0 += n_kv;
+                continue;
+            }
+
+            // Epilogue: O/l, L = m + log l, tO = (T - r (O/l)) / l, once the item's last value MMAs are complete
+            // (which implies all earlier ones)
             const int g_last = g0 + n_kv - 1;
-            if (n_kv >= 2) ok = mbar_wait_warp(smem_u32(&bar_pv_done), (g_last - 1) & 1, abort_state);
-            if (ok) ok = mbar_wait_warp(smem_u32(&bar_pv_done), g_last & 1, abort_state);
+            ok = mbar_wait_warp(smem_u32(&bar_pv_done[g_last & 1]), (g_last >> 1) & 1, abort_state);
+            if (ok && kGroups == 2) {
+                // the other group's sums, brought to the final reference (it last knew m_other; 0 if it had no tile)
+                ok = mbar_wait_warp(finbar, it & 1, abort_state);
+                if (ok) {
+                    const float f = ex2f(m_other - m_ref);
+                    l_run = fmaf(ld_shared_f32(xch_l), f, l_run);
+                    r_run = fmaf(ld_shared_f32(xch_r), f, r_run);
+                }
+            }
             if (!ok) break;
             tc_fence_after();
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
@@ -1072,15 +1221,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // layout of the output tensor maps (row r, 16-byte chunk c of a 64-column half at r*128 + (c ^ (r&7))*16)
             uint32_t stage_o = 0, stage_t = 0;
             if (kStageSlots > 0) {
-                // Ring positions of this item: 2 n_kv tiles, plus the previous item's staging slots.  Its own staging
-                // slots come after the next item's leading K tiles (every item has n_kv tiles here: the kernel that
-                // cuts the keys into chunks stages nothing), or right after its last V tile if it is the CTA's last.
-                const bool has_next = n_items - item > static_cast<int>(gridDim.x);
-                const int next_start = (ring_slot + 2 * (n_kv % kSlots) + (it > 0 ? kStageSlots : 0)) % kSlots;
-                const int so = has_next ? (next_start + min(2, n_kv)) % kSlots : next_start;
-                stage_o = smem_ring + so * Plan::kSlotBytes + row * 128;
-                stage_t = smem_ring + ((so + 1) % kSlots) * Plan::kSlotBytes + row * 128;
-                ring_slot = next_start;
+                stage_o = smem_ring + stage_slot_o * Plan::kSlotBytes + row * 128;
+                stage_t = smem_ring + ((stage_slot_o + 1) % kSlots) * Plan::kSlotBytes + row * 128;
             }
 #pragma unroll 1
             for (int c0 = 0; c0 < D; c0 += 32) {

@@ -1,0 +1,100 @@
+"""In-kernel timeline of one CTA (debugging aid; not used by the library's normal operation).
+
+Builds a second copy of the library with -DATTN_JVP_TRACE=2 (clock64 stamps at the hand-over points of the
+roles of one CTA, see attn_jvp_kernel.cuh), runs one shape through it and prints, per 64-key tile, when the MMA
+warp issued the score and value MMAs and when the softmax warps saw the scores, agreed on the reference max,
+stored P~ and handed the tile back -- plus the mean tile period.  The cycle figures quoted in the design doc and
+profiles/ come from this tool:
+
+    python -m paper_2510_08431_b200.trace --B 1 --H 8 --Lq 18944 --Lk 4096 --D 128 [--mode jvp|kv_free|fwd] [--groups 1|2]
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+import torch
+
+from . import attn_jvp as binding
+from . import build as lib_build
+from . import synth
+
+TRACE_LIB = os.path.join(lib_build.PKG, "libattn_jvp_trace.so")
+EVENTS, STEPS = 32, 96
+
+
+def build_trace_library() -> str:
+    stale = (not os.path.exists(TRACE_LIB)) or any(os.path.getmtime(d) > os.path.getmtime(TRACE_LIB) for d in lib_build.DEPS)
+    if stale:
+        cmd = [lib_build._nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+               "-DATTN_JVP_TRACE=2", "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(lib_build.ROOT, "include"),
+               "-o", TRACE_LIB, lib_build.SRC, "-lcudart"]
+        subprocess.run(cmd, check=True, capture_output=True)
+    return TRACE_LIB
+
+
+def run(B, H, Lq, Lk, D, mode="jvp", groups=0, first=20, count=6, seed=4):
+    """Runs the shape three times through the trace build and returns the [EVENTS][STEPS] stamp array."""
+    lib = ctypes.CDLL(build_trace_library())
+    x = synth.make_inputs(B, H, Lq, Lk, D, 1.0, 0.5, seed, kv_tangent_free=(mode != "jvp"))
+    g = {k: (None if t is None else t.cuda()) for k, t in x.items()}
+    flags = {"jvp": 0, "kv_free": binding.KV_TANGENT_FREE, "fwd": binding.FWD_ONLY}[mode]
+    lib.attn_jvp_set_tuning(binding.TUNE_SOFTMAX_GROUPS, int(groups))
+    o = torch.empty_like(g["q"]); to = torch.empty_like(g["q"])
+    lse = torch.empty((B, H, Lq), dtype=torch.float32, device="cuda")
+    vp = ctypes.c_void_p
+    lib.attn_jvp_fwd_stream.argtypes = [vp] * 9 + [ctypes.c_int] * 5 + [ctypes.c_float, ctypes.c_uint, vp]
+    p = lambda t: None if t is None else t.data_ptr()
+    for _ in range(3):
+        rc = lib.attn_jvp_fwd_stream(p(g["q"]), p(g["k"]), p(g["v"]), p(g["tq"]), p(g["tk"]), p(g["tv"]), p(o), p(to),
+                                     p(lse), B, H, Lq, Lk, D, D ** -0.5, flags, torch.cuda.current_stream().cuda_stream)
+        assert rc == 0, rc
+    torch.cuda.synchronize()
+    assert lib.attn_jvp_device_status() == 0
+    buf = (ctypes.c_longlong * (EVENTS * STEPS))()
+    lib.attn_jvp_debug_read_trace.argtypes = [vp, ctypes.c_int]
+    assert lib.attn_jvp_debug_read_trace(buf, EVENTS * STEPS) == EVENTS * STEPS
+    return np.array(buf, dtype=np.int64).reshape(EVENTS, STEPS)
+
+
+NAMES = {21: "MMA   score MMAs: issue begins", 2: "MMA   score MMAs issued", 3: "MMA   value MMAs: issue begins",
+         4: "MMA   value MMAs issued", 29: "MMA   burst begins (loop top)", 30: "MMA   after tensor-core fence",
+         23: "MMA   burst issued, warp reconverged", 22: "MMA   blocks for the tile's barriers", 24: "MMA   blocks for H~",
+         5: "  softmax scores seen (s_full)", 26: "  softmax scores in registers", 27: "  softmax reference max agreed",
+         28: "  softmax P~ stored", 13: "  softmax tile handed back"}
+
+
+def report(t, first=20, count=6):
+    ev = [(t[e][g], nm, g) for e, nm in NAMES.items() for g in range(first, first + count) if t[e][g] > 0]
+    ev.sort()
+    base = ev[0][0] if ev else 0
+    for tm, nm, g in ev:
+        print(f"{tm - base:8d}  {nm} (tile {g})")
+    pv = t[3][10:60]
+    pv = pv[pv > 0]
+    if len(pv) > 1:
+        print(f"mean tile period (value-MMA issue, tiles 10..{9 + len(pv)}): {(pv[-1] - pv[0]) / (len(pv) - 1):.0f} cycles")
+    sm = (t[13][10:60] - t[5][10:60])[(t[13][10:60] > 0) & (t[5][10:60] > 0)]
+    if len(sm):
+        print(f"softmax warp, scores seen -> tile handed back: mean {sm.mean():.0f} cycles")
+    print("MMA warp had to block for a tile:", int((t[22][10:60] > 0).sum()), "of 50 tiles; CTA lifetime",
+          int(t[EVENTS - 1][1] - t[EVENTS - 1][0]), "cycles")
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--B", type=int, default=1); ap.add_argument("--H", type=int, default=8)
+    ap.add_argument("--Lq", type=int, default=128 * 148); ap.add_argument("--Lk", type=int, default=4096)
+    ap.add_argument("--D", type=int, default=128)
+    ap.add_argument("--mode", default="jvp", choices=["jvp", "kv_free", "fwd"])
+    ap.add_argument("--groups", type=int, default=0)
+    ap.add_argument("--first", type=int, default=20); ap.add_argument("--count", type=int, default=4)
+    a = ap.parse_args()
+    report(run(a.B, a.H, a.Lq, a.Lk, a.D, a.mode, a.groups), a.first, a.count)
+
+
+if __name__ == "__main__":
+    main()
