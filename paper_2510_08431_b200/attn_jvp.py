@@ -89,6 +89,9 @@ def load():
             forced = os.environ.get("ATTN_JVP_SOFTMAX_GROUPS")
             if forced:
                 lib.attn_jvp_set_tuning(TUNE_SOFTMAX_GROUPS, int(forced))
+            forced = os.environ.get("ATTN_JVP_CTA_PAIR")
+            if forced:
+                lib.attn_jvp_set_tuning(TUNE_CTA_PAIR, int(forced))
             _lib = lib
     return _lib
 
@@ -110,6 +113,7 @@ def attn_jvp_version() -> int:
 
 
 TUNE_SOFTMAX_GROUPS = 1
+TUNE_CTA_PAIR = 2
 
 
 def attn_jvp_debug_timeout_info():

@@ -40,6 +40,7 @@ struct DeviceState {
     std::atomic<int*> host_status_dev{nullptr};   // ... and its device-side address (published first)
     std::atomic<bool> unwatched_launch{false};    // a kernel ran here before the status word existed
     std::atomic<int> dyn_smem[2][3][2][2];        // dynamic shared memory per kernel instantiation, 0 = not set up
+    std::atomic<int> dyn_smem_pair[2];            // ... of the CTA-pair kernels
     std::atomic<void*> static_scratch{nullptr};   // device address of the built-in scratch array
 };
 DeviceState g_dev[kMaxDevices];
@@ -48,6 +49,25 @@ std::atomic<EncodeTiledFn> g_encode_tiled{nullptr};
 
 // Tuning knobs (attn_jvp_set_tuning); 0 = the library's own choice.
 std::atomic<int> g_tune_softmax_groups{0};
+std::atomic<int> g_tune_cta_pair{0};
+
+// Softmax groups of the CTA-pair kernel (measured: one group is 3-8 % faster than two there as well).
+int softmax_groups_for_pair() {
+    const int forced = g_tune_softmax_groups.load(std::memory_order_relaxed);
+    return forced == 2 ? 2 : 1;
+}
+
+// Whether a call runs on the CTA-pair kernel (clusters of two CTAs sharing the K/V operand tiles and one MMA
+// instruction stream).  It exists for the full JVP at D = 128.
+bool use_cta_pair(int mode, int D, bool split, int tiles_per_item) {
+    if (mode != attn_jvp::kModeJvp || D != 128 || split) return false;
+    const int forced = g_tune_cta_pair.load(std::memory_order_relaxed);
+    if (forced == 1) return false;
+    if (forced == 2) return true;
+    // Measured on B200: 4-20 % faster than one CTA per query tile from about eight key tiles per item on (12 % on
+    // the 32760-token self-attention workloads), 4 % slower with two key tiles per item.
+    return tiles_per_item >= 6;
+}
 
 // Softmax warpgroups per CTA for a kernel variant: two groups take alternate key tiles, which pays where the
 // softmax arithmetic, not the tensor pipe, sets the pace of a key tile.
@@ -151,11 +171,11 @@ bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
     return a0 < b0 + nb && b0 < a0 + na;
 }
 
-template <int D, int MODE, bool SPLIT, int GROUPS>
+template <int D, int MODE, bool SPLIT, int GROUPS, bool PAIR = false>
 int launch(const CUtensorMap* maps, const KernelArgs& ka, dim3 grid, cudaStream_t stream, DeviceState& st) {
-    auto kern = attn_jvp::attn_jvp_fwd_kernel<D, MODE, SPLIT, GROUPS>;
+    auto kern = attn_jvp::attn_jvp_fwd_kernel<D, MODE, SPLIT, GROUPS, PAIR>;
     using Plan = attn_jvp::SmemPlan<D, GROUPS>;
-    std::atomic<int>& slot = st.dyn_smem[D == 128][MODE][SPLIT][GROUPS - 1];
+    std::atomic<int>& slot = PAIR ? st.dyn_smem_pair[GROUPS - 1] : st.dyn_smem[D == 128][MODE][SPLIT][GROUPS - 1];
     int smem = slot.load(std::memory_order_acquire);
     if (smem == 0) {
         // dynamic shared memory = the operand layout (declared 1024-byte aligned in the kernel) plus the exchange
@@ -179,8 +199,27 @@ int launch(const CUtensorMap* maps, const KernelArgs& ka, dim3 grid, cudaStream_
             slot.store(want, std::memory_order_release);
         }
     }
+    if (PAIR) {
+        // clusters of two CTAs (the two SMs of a TPC); the grid holds an even number of CTAs
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = grid;
+        cfg.blockDim = dim3(attn_jvp::num_threads(GROUPS), 1, 1);
+        cfg.dynamicSmemBytes = (size_t)smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, kern, maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], maps[6],
+                                           maps[7], maps[8], ka);
+        if (e != cudaSuccess) return cuda_fail("cluster kernel launch", e);
+        return 0;
+    }
     kern<<<grid, attn_jvp::num_threads(GROUPS), smem, stream>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], maps[6],
-                                                     maps[7], ka);
+                                                     maps[7], maps[8], ka);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail("kernel launch", e);
     return 0;
@@ -267,7 +306,7 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     cudaError_t e;
 
     // ---- tensor maps (Q-side boxes are 128 rows, K-side boxes 64 rows) ----
-    CUtensorMap maps[8];
+    CUtensorMap maps[9];
     if (int rc = make_map(&maps[0], q, B, Lq, H, D, attn_jvp::kBlockM)) return rc;
     if (int rc = make_map(&maps[1], k, B, Lk, H, D, attn_jvp::kBlockN)) return rc;
     if (int rc = make_map(&maps[2], v, B, Lk, H, D, attn_jvp::kBlockN)) return rc;
@@ -277,6 +316,8 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     // output tiles (bf16, stored from shared memory by TMA; the split-KV kernel does not use these two)
     if (int rc = make_map(&maps[6], o, B, Lq, H, D, attn_jvp::kBlockM)) return rc;
     if (int rc = make_map(&maps[7], fwd_only ? o : to, B, Lq, H, D, attn_jvp::kBlockM)) return rc;
+    // K once more with boxes of half a key tile (the CTA-pair kernel splits the operand of tQ K^T by rows)
+    if (int rc = make_map(&maps[8], k, B, Lk, H, D, attn_jvp::kBlockN / 2)) return rc;
 
     KernelArgs ka;
     ka.o = reinterpret_cast<__nv_bfloat16*>(o);
@@ -312,9 +353,22 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     // round-robin costs up to one item of imbalance at the end, which is more than the overlap saves there).
     const int tiles_per_item = split ? tiles_per_split : ka.n_kv_tiles;
     const bool persistent = tiles_per_item <= kPersistentMaxTiles;
+    int rc;
+    if (use_cta_pair(mode, D, split, tiles_per_item)) {
+        // A work item is a 256-row query block (two tiles, one per CTA of a pair); with an odd number of tiles the
+        // last pair's second CTA has no rows and writes nothing.
+        const long long n_q_pairs = (n_q_tiles + 1) / 2;
+        const long long n_pair_items = n_q_pairs * H * B;
+        ka.n_q_tiles = (int)n_q_pairs;
+        ka.n_items = (int)n_pair_items;
+        const long long max_pairs = st.sm_count / 2;
+        const long long n_pairs = (persistent && n_pair_items > max_pairs) ? max_pairs : n_pair_items;
+        const dim3 pair_grid((unsigned)(2 * n_pairs), 1, 1);
+        if (softmax_groups_for_pair() == 2) return launch<128, attn_jvp::kModeJvp, false, 2, true>(maps, ka, pair_grid, stream, st);
+        return launch<128, attn_jvp::kModeJvp, false, 1, true>(maps, ka, pair_grid, stream, st);
+    }
     const long long n_ctas = (persistent && n_items > st.sm_count) ? st.sm_count : n_items;
     const dim3 grid((unsigned)n_ctas, 1, 1);
-    int rc;
     const int groups = softmax_groups_for(mode, D);
 #define ATTN_JVP_DISPATCH_G(DD, SS, GG)                                                                            \
     switch (mode) {                                                                                               \
@@ -680,6 +734,10 @@ int attn_jvp_selftest_bounded_wait(void* cuda_stream) {
 int attn_jvp_set_tuning(int knob, int value) {
     if (knob == ATTN_JVP_TUNE_SOFTMAX_GROUPS && value >= 0 && value <= 2) {
         g_tune_softmax_groups.store(value, std::memory_order_relaxed);
+        return 0;
+    }
+    if (knob == ATTN_JVP_TUNE_CTA_PAIR && value >= 0 && value <= 2) {
+        g_tune_cta_pair.store(value, std::memory_order_relaxed);
         return 0;
     }
     return ATTN_JVP_ERR_FLAGS;

@@ -267,19 +267,79 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// ---- CTA pair (cluster of two CTAs on the two SMs of a TPC, one tcgen05.mma feeding both) ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+// Arrival on a barrier of another CTA of the cluster.  What is handed over with it lives in tensor memory and is
+// ordered by the tcgen05 fences on both sides; a cluster-scope release on the arrival itself was measured to cost
+// about a thousand cycles per arrival and is not needed for that.
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void st_shared_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+// Barrier over all threads of the cluster.  Every thread of both CTAs reaches each of its uses on every path
+// (all other waits in the kernel are bounded), so it cannot be left waiting.
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA tile load of a CTA pair: the data lands in this CTA's shared memory, the bytes are counted on a barrier that
+// may live in the pair's other CTA (`bar` is a shared::cluster address).  No multicast: each CTA fetches its own.
+__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                                 int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
+// completion of all earlier MMAs of this thread, signalled on the barrier at this address in BOTH CTAs of the pair
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(static_cast<uint16_t>(3)) : "memory");
+}
+template <bool kAccumulate>
+__device__ __forceinline__ void mma_ss_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+    if (kAccumulate) {
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.u32 p, 1, 1;\n\t"
+                     "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc) : "memory");
+    } else {
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, 1, 1;\n\t"
+                     "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc) : "memory");
+    }
+}
+__device__ __forceinline__ void mma_ts_pair(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
 // Instruction descriptor for kind::f16: bf16 x bf16 -> fp32, M = 128.
-__host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major) {
+__host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major, int m = kBlockM) {
     return (1u << 4)                       // accumulator format: fp32
          | (1u << 7)                       // A format: bf16
          | (1u << 10)                      // B format: bf16
          | (0u << 15)                      // A: K-major
          | ((b_mn_major ? 1u : 0u) << 16)  // B: K-major or MN-major
          | (static_cast<uint32_t>(n >> 3) << 17)
-         | (static_cast<uint32_t>(kBlockM >> 4) << 24);
+         | (static_cast<uint32_t>(m >> 4) << 24);
 }
 
 // Shared-memory matrix descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
@@ -399,13 +459,20 @@ __host__ __device__ constexpr int score_buffers(int D, int mode) {
     return ((mode == kModeFwdOnly ? D : 2 * D) <= 128) ? 3 : 2;
 }
 
-template <int D, int MODE, bool kSplit, int kGroups>
+// kPair: the kernel is launched in clusters of two CTAs that share every work item -- a 256-row query block of
+// which each CTA owns 128 rows (its own Q, tQ, softmax warps, accumulators and outputs).  The MMA warp of the
+// cluster's first CTA issues every tcgen05.mma for both (cta_group::2, M = 256): the B operands (K, tK, V, tV
+// tiles) are split between the two CTAs' shared memories, each CTA loading its part through its own TMA
+// requests (no multicast), and one instruction stream feeds two tensor pipes.  tm_k32 (32-row boxes of K) is
+// only used by that variant.
+template <int D, int MODE, bool kSplit, int kGroups, bool kPair>
 __global__ void __launch_bounds__(num_threads(kGroups), 1)
 attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_tq,
                     const __grid_constant__ CUtensorMap tm_tk, const __grid_constant__ CUtensorMap tm_tv,
                     const __grid_constant__ CUtensorMap tm_o, const __grid_constant__ CUtensorMap tm_to,
-                    const KernelArgs args) {
+                    const __grid_constant__ CUtensorMap tm_k32, const KernelArgs args) {
+    static_assert(!kPair || (MODE == kModeJvp && D == 128 && !kSplit), "the CTA-pair variant exists for the full JVP at D = 128");
     using Plan = SmemPlan<D, kGroups>;
     constexpr int kFirstSoftmaxWarp = first_softmax_warp(kGroups);
     constexpr int kHalves = Plan::kHalves;
@@ -420,7 +487,16 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // MMAs -> score MMAs: there P~ is handed to the MMA warp as soon as it is stored, and the MMAs that read it run
     // beside the H~ arithmetic (H~ follows through a barrier of its own).  In the full mode the MMA warp never
     // waits for the softmax warps, and the second hand-over would only add work (measured: 1 % slower).
-    constexpr bool kSplitHandover = kHasTQ && !kHasTKV;
+    // The CTA pair runs at the pace of the chain score MMAs -> softmax -> value MMAs as well (one instruction stream
+    // feeds two tensor pipes, so the issuing warp is no longer what a key tile waits for).  Option: it hands P~
+    // over early too, and its softmax warps start on S while the MMAs of tQ K^T are still running (kEarlyS: the
+    // scores are published in two steps, S after the stacked chain, tS after the second one).
+    // (Measured with one softmax group: 6 % slower than the plain hand-over, because there the softmax warps'
+    // throughput, not their latency, sets the pace, and the extra wait and fence lengthen their tile.  Kept as a
+    // compile-time option.)
+    constexpr bool kEarlyHandover = false;
+    constexpr bool kSplitHandover = kHasTQ && (!kHasTKV || (kPair && kEarlyHandover));
+    constexpr bool kEarlyS = kPair && kHasTQ && kGroups == 1 && kEarlyHandover;
     constexpr int kBufs = score_buffers(D, MODE);            // score buffers = how many tiles the score MMAs run ahead
     constexpr int kScoreCol0 = (kBufs == 3) ? 128 : 256;     // first column of score buffer 0
     static_assert(kScoreCol0 + kBufs * kScoreBufStride <= kTmemCols, "score buffers must fit into tensor memory");
@@ -433,6 +509,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     __shared__ __align__(8) uint64_t bar_slot_full[kSlots];
     __shared__ __align__(8) uint64_t bar_slot_empty[kSlots];
     __shared__ __align__(8) uint64_t bar_s_full[kBufs];
+    __shared__ __align__(8) uint64_t bar_ts_full[kBufs];    // kEarlyS: tS of the tile is complete (bar_s_full then means S alone)
     __shared__ __align__(8) uint64_t bar_p_full[kBufs];     // P~ of the tile is in tensor memory
     __shared__ __align__(8) uint64_t bar_h_full[kBufs];     // H~ of the tile is in tensor memory (some 500 cycles later)
     __shared__ __align__(8) uint64_t bar_pv_done[2];        // the value MMAs of tile g (and all before) are complete: [g & 1]
@@ -443,22 +520,28 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // two softmax groups, one barrier per quarter of the rows (a pair of warps, one of each group):
     __shared__ __align__(8) uint64_t bar_m[4];          // the reference max after tile g is published (phase g & 1)
     __shared__ __align__(8) uint64_t bar_fin[4];        // the non-finishing group's partial l, r of the item are published
+    __shared__ __align__(8) uint64_t bar_fin_read[4];   // ... and have been read by the finishing group
     __shared__ uint32_t tmem_base_smem;
     __shared__ int cta_abort;
 
     const int warp = __shfl_sync(0xffffffffu, threadIdx.x >> 5, 0);   // warp-uniform by construction
     const int lane = threadIdx.x & 31;
 #ifdef ATTN_JVP_TRACE
-    const bool trace_on = blockIdx.x == gridDim.x / 2;
+    const bool trace_on = blockIdx.x == (kPair ? (gridDim.x / 4) * 2 : gridDim.x / 2);
 #endif
 
     // A CTA is persistent: it walks the work items blockIdx.x, blockIdx.x + gridDim.x, ... in the same order in
     // every role.  An item is one 128-row query tile of one (batch, head[, key chunk]); query tiles vary fastest
     // so that the CTAs running at one time share one head's K/V in L2.
+    // CTA pair: both CTAs walk the same items (one item = two query tiles); this CTA's rank picks its rows.
+    const uint32_t cta_rank = kPair ? cluster_ctarank() : 0u;
+    const bool lead_cta = cta_rank == 0u;
+    const int first_item = kPair ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+    const int item_stride = kPair ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
     struct Item { int q0, h, b, split, tile0, n_kv; };
     auto decode = [&](int item) -> Item {
         Item w;
-        w.q0 = (item % args.n_q_tiles) * kBlockM;
+        w.q0 = (item % args.n_q_tiles) * (kPair ? 2 * kBlockM : kBlockM) + static_cast<int>(cta_rank) * kBlockM;
         const int rest = item / args.n_q_tiles;
         w.h = rest % args.H;
         const int z = rest / args.H;
@@ -474,9 +557,12 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
     // An earlier CTA of this (or a previous) launch gave up: do not start.  One thread reads
     // the flag so that the whole CTA takes the same decision.
-    if (threadIdx.x == 0) cta_abort = *reinterpret_cast<volatile int*>(&g_abort_flag);
-    __syncthreads();
-    if (cta_abort != 0) return;
+    // (A CTA pair takes this decision together, after its barriers are set up: see below.)
+    if (!kPair) {
+        if (threadIdx.x == 0) cta_abort = *reinterpret_cast<volatile int*>(&g_abort_flag);
+        __syncthreads();
+        if (cta_abort != 0) return;
+    }
 
 #ifdef ATTN_JVP_TRACE
     if (trace_on && threadIdx.x == 0) g_trace[kTraceEvents - 1][0] = clock64();      // CTA begins
@@ -509,18 +595,21 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         for (int i = 0; i < kBufs; ++i) {
             mbar_init(smem_u32(&bar_s_full[i]), 1);
-            mbar_init(smem_u32(&bar_p_full[i]), kSoftmaxThreads / 32);    // one arrival per softmax warp
-            mbar_init(smem_u32(&bar_h_full[i]), kSoftmaxThreads / 32);
+            mbar_init(smem_u32(&bar_ts_full[i]), 1);
+            // one arrival per softmax warp of the tile's group (CTA pair: of both CTAs, on the first CTA's barrier)
+            mbar_init(smem_u32(&bar_p_full[i]), (kPair ? 2 : 1) * kSoftmaxThreads / 32);
+            mbar_init(smem_u32(&bar_h_full[i]), (kPair ? 2 : 1) * kSoftmaxThreads / 32);
         }
         mbar_init(smem_u32(&bar_pv_done[0]), 1);
         mbar_init(smem_u32(&bar_pv_done[1]), 1);
-        mbar_init(smem_u32(&bar_acc_free), kSoftmaxThreads / 32);
+        mbar_init(smem_u32(&bar_acc_free), (kPair ? 2 : 1) * kSoftmaxThreads / 32);
         mbar_init(smem_u32(&bar_drain), 1);
         mbar_init(smem_u32(&bar_stage_ready), 1);
         mbar_init(smem_u32(&bar_stage_full), kSoftmaxThreads / 32);
         for (int i = 0; i < 4; ++i) {
             mbar_init(smem_u32(&bar_m[i]), 1);
             mbar_init(smem_u32(&bar_fin[i]), 1);
+            mbar_init(smem_u32(&bar_fin_read[i]), 1);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 #ifdef ATTN_JVP_DEBUG
@@ -532,10 +621,29 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
 #endif
     }
+    if (kPair) {
+        // The pair decides together whether to run at all (an earlier CTA gave up): the first CTA reads the flag
+        // and writes it into both CTAs; the cluster barrier also makes both CTAs' barriers visible to each other
+        // before anything arrives on them from the other side.
+        if (threadIdx.x == 0 && lead_cta) {
+            const int flag = *reinterpret_cast<volatile int*>(&g_abort_flag);
+            cta_abort = flag;
+            st_shared_cluster_u32(map_to_cta(smem_u32(&cta_abort), 1u), static_cast<uint32_t>(flag));
+        }
+        cluster_sync_all();
+        if (*reinterpret_cast<volatile int*>(&cta_abort) != 0) return;
+    }
     if (warp == kMmaWarp) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&tmem_base_smem)), "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        // (pair: the same warp of both CTAs allocates, each in its own SM's tensor memory; both get column 0)
+        if (kPair) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(&tmem_base_smem)), "r"(kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(&tmem_base_smem)), "r"(kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     if (warp == kProducerWarp && lane == 0) {
         prefetch_tensormap(&tm_q);
@@ -545,6 +653,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (kHasTKV) { prefetch_tensormap(&tm_tk); prefetch_tensormap(&tm_tv); }
         if (kStageSlots > 0) prefetch_tensormap(&tm_o);
         if (kStageSlots > 1) prefetch_tensormap(&tm_to);
+        if (kPair) prefetch_tensormap(&tm_k32);
     }
     tc_fence_before();
     __syncthreads();
@@ -576,7 +685,13 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             constexpr uint32_t kQTx = (kHasTQ ? 2u : 1u) * Plan::kQBytes;
             constexpr uint32_t kKTx = (kHasTKV ? 2u : 1u) * kHalves * Plan::kKvHalfBytes;
             constexpr uint32_t kVTx = kKTx;
-            const uint32_t qbar = smem_u32(&bar_q_full);
+            // CTA pair: the `full` barriers that count, the MMA-issuing warp's, are the first CTA's; both CTAs' loads
+            // report their bytes there and the first CTA's producer announces the bytes of both.
+            const uint32_t qbar = kPair ? map_to_cta(smem_u32(&bar_q_full), 0u) : smem_u32(&bar_q_full);
+            // pair: offset of the second operand region of a ring slot (the halves of K / V that the N = 64 and
+            // N = 128 MMAs take from each CTA at a common offset)
+            constexpr uint32_t kPairRegionB = kHalves * Plan::kKvHalfBytes;   // 16 KB at D = 128
+            static_assert(!kPair || kPairRegionB == 16384, "pair layout is laid out for D = 128");
             // ring position: slot, the parity of the slot's `full` phase that this lap completes, and whether the
             // ring has been round once (before that the slots are empty without anybody saying so)
             int r_slot = 0;
@@ -591,7 +706,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (!mbar_wait(smem_u32(&bar_slot_empty[slot]), r_parity ^ 1u, abort_state)) return false;
                 }
                 slot_addr = smem_ring + slot * Plan::kSlotBytes;
-                bar = smem_u32(&bar_slot_full[slot]);
+                bar = kPair ? map_to_cta(smem_u32(&bar_slot_full[slot]), 0u) : smem_u32(&bar_slot_full[slot]);
                 TRACE(0, slot);       // producer: slot acquired, loads issued next
                 if (++r_slot == kSlots) { r_slot = 0; r_parity ^= 1u; r_lapped = true; }
                 return true;
@@ -600,6 +715,21 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 int slot;
                 uint32_t dst, bar;
                 if (!acquire(slot, dst, bar)) return false;
+                if (kPair) {
+                    // The stacked operand [K ; tK] is split by tensor: this CTA holds K (first CTA) or tK (second) as
+                    // [half 0 (8 KB)][half 1 (8 KB)].  The N = 64 operand of tQ K^T is split by rows: K rows
+                    // 32 r .. 32 r + 31 as [half 0 (4 KB)][half 1 (4 KB)] in the slot's second region.
+                    constexpr uint32_t kTxPerCta = 2 * Plan::kKvHalfBytes + Plan::kKvHalfBytes;     // 16 KB + 8 KB
+                    if (lead_cta) mbar_arrive_expect_tx(smem_u32(&bar_slot_full[slot]), 2 * kTxPerCta);
+                    const int row0 = (w.tile0 + j) * kBlockN;
+#pragma unroll
+                    for (int hf = 0; hf < kHalves; ++hf) {
+                        tma_load_4d_pair(dst + hf * Plan::kKvHalfBytes, lead_cta ? &tm_k : &tm_tk, bar, hf * 64, w.h, row0, w.b);
+                        tma_load_4d_pair(dst + kPairRegionB + hf * (Plan::kKvHalfBytes / 2), &tm_k32, bar, hf * 64, w.h,
+                                         row0 + 32 * static_cast<int>(cta_rank), w.b);
+                    }
+                    return true;
+                }
                 mbar_arrive_expect_tx(bar, kKTx);
                 // per 64-column half: [K_half (8 KB)][tK_half (8 KB)] so that [K ; tK] is one N = 128 operand
 #pragma unroll
@@ -614,6 +744,18 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 int slot;
                 uint32_t dst, bar;
                 if (!acquire(slot, dst, bar)) return false;
+                if (kPair) {
+                    // [V | tV] is split by tensor: this CTA holds V (first CTA) or tV (second) as two 64-wide N atoms.
+                    // The N = 128 operand of H~ V is split by columns: V atom r in the slot's second region.
+                    constexpr uint32_t kTxPerCta = 2 * Plan::kKvHalfBytes + Plan::kKvHalfBytes;
+                    if (lead_cta) mbar_arrive_expect_tx(smem_u32(&bar_slot_full[slot]), 2 * kTxPerCta);
+                    const int row0 = (w.tile0 + j) * kBlockN;
+#pragma unroll
+                    for (int hf = 0; hf < kHalves; ++hf)
+                        tma_load_4d_pair(dst + hf * Plan::kKvHalfBytes, lead_cta ? &tm_v : &tm_tv, bar, hf * 64, w.h, row0, w.b);
+                    tma_load_4d_pair(dst + kPairRegionB, &tm_v, bar, 64 * static_cast<int>(cta_rank), w.h, row0, w.b);
+                    return true;
+                }
                 mbar_arrive_expect_tx(bar, kVTx);
                 // [V_half0][V_half1][tV_half0][tV_half1]: consecutive 64-wide N atoms of [V | tV]
 #pragma unroll
@@ -634,6 +776,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 TRACE(17, stage_it);  // producer: staged tiles complete, stores issued next
 #pragma unroll
                 for (int hf = 0; hf < kHalves; ++hf) {
+                    if (kPair && stage_w.q0 >= args.Lq) break;     // second CTA of a pair whose rows all lie past Lq
                     tma_store_4d(&tm_o, smem_ring + stage_slot[0] * Plan::kSlotBytes + hf * Plan::kQHalfBytes,
                                  hf * 64, stage_w.h, stage_w.q0, stage_w.b);
                     if (kStageSlots > 1)
@@ -654,7 +797,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 for (int s = 0; s < kStageSlots; ++s) {
                     uint32_t dst, bar;
                     if (!acquire(stage_slot[s], dst, bar)) return false;
-                    mbar_arrive(bar);
+                    if (!kPair || lead_cta) mbar_arrive(smem_u32(&bar_slot_full[stage_slot[s]]));
                 }
                 mbar_arrive(smem_u32(&bar_stage_ready));
                 TRACE(9, of_it);      // producer: staging slots handed over
@@ -665,22 +808,31 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             };
             Item prev_w{};
             int it = 0;
-            for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
+            for (int item = first_item; ok && item < n_items; item += item_stride, ++it) {
                 w = decode(item);
                 if (it > 0) ok = mbar_wait(smem_u32(&bar_q_free), (it - 1) & 1, abort_state);
                 if (!ok) break;
                 TRACE(1, it);         // producer: Q, tQ may be replaced
-                mbar_arrive_expect_tx(qbar, kQTx);
+                if (kPair) {
+                    if (lead_cta) mbar_arrive_expect_tx(smem_u32(&bar_q_full), 2 * kQTx);
 #pragma unroll
-                for (int hf = 0; hf < kHalves; ++hf) {
-                    tma_load_4d(smem_q + hf * Plan::kQHalfBytes, &tm_q, qbar, hf * 64, w.h, w.q0, w.b);
-                    if (kHasTQ) tma_load_4d(smem_tq + hf * Plan::kQHalfBytes, &tm_tq, qbar, hf * 64, w.h, w.q0, w.b);
+                    for (int hf = 0; hf < kHalves; ++hf) {
+                        tma_load_4d_pair(smem_q + hf * Plan::kQHalfBytes, &tm_q, qbar, hf * 64, w.h, w.q0, w.b);
+                        tma_load_4d_pair(smem_tq + hf * Plan::kQHalfBytes, &tm_tq, qbar, hf * 64, w.h, w.q0, w.b);
+                    }
+                } else {
+                    mbar_arrive_expect_tx(qbar, kQTx);
+#pragma unroll
+                    for (int hf = 0; hf < kHalves; ++hf) {
+                        tma_load_4d(smem_q + hf * Plan::kQHalfBytes, &tm_q, qbar, hf * 64, w.h, w.q0, w.b);
+                        if (kHasTQ) tma_load_4d(smem_tq + hf * Plan::kQHalfBytes, &tm_tq, qbar, hf * 64, w.h, w.q0, w.b);
+                    }
                 }
-                const bool has_next = n_items - item > static_cast<int>(gridDim.x);
+                const bool has_next = n_items - item > item_stride;
                 if (has_next) {
                     // the next item's Q, tQ can only be loaded once this item's score MMAs are done: have them
                     // waiting in L2 by then
-                    const Item nx = decode(item + gridDim.x);
+                    const Item nx = decode(item + item_stride);
 #pragma unroll
                     for (int hf = 0; hf < kHalves; ++hf) {
                         tma_prefetch_4d(&tm_q, hf * 64, nx.h, nx.q0, nx.b);
@@ -726,17 +878,19 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
             }
         }
-    } else if (warp == kMmaWarp) {
+    } else if (warp == kMmaWarp && lead_cta) {
         // =====================================================================================
-        // MMA issuer.  The whole warp walks the loop in lock step, so that addresses, descriptors and
+        // MMA issuer (CTA pair: of the first CTA only, for both).  The whole warp walks the loop in lock step, so that addresses, descriptors and
         // loop state stay warp-uniform; one elected lane issues every tcgen05.mma and the commits
         // that track them.
         // =====================================================================================
         {
-            constexpr uint32_t kIdescS1 = make_idesc(kHasTKV ? 2 * kBlockN : kBlockN, false);  // Q x [K;tK] or Q x K
-            constexpr uint32_t kIdescS2 = make_idesc(kBlockN, false);                          // tQ x K
-            constexpr uint32_t kIdescPV = make_idesc(kHasTKV ? 2 * D : D, true);               // P~ x [V|tV] or P~ x V
-            constexpr uint32_t kIdescHV = make_idesc(D, true);                                 // H~ x V
+            // (CTA pair: M = 256, 128 rows in each CTA; N counts the columns of both CTAs' parts of the B operand)
+            constexpr int kMmaM = kPair ? 2 * kBlockM : kBlockM;
+            constexpr uint32_t kIdescS1 = make_idesc(kHasTKV ? 2 * kBlockN : kBlockN, false, kMmaM);  // Q x [K;tK] or Q x K
+            constexpr uint32_t kIdescS2 = make_idesc(kBlockN, false, kMmaM);                          // tQ x K
+            constexpr uint32_t kIdescPV = make_idesc(kHasTKV ? 2 * D : D, true, kMmaM);               // P~ x [V|tV] or P~ x V
+            constexpr uint32_t kIdescHV = make_idesc(D, true, kMmaM);                                 // H~ x V
             constexpr uint32_t kVLbo = Plan::kKvHalfBytes;   // bytes between 64-wide N atoms of a V slot
             const bool leader = elect_one();
             bool ok = true;
@@ -766,29 +920,51 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             auto prepare_v = [&](int slot) { v_lo = make_desc_lo(smem_ring + slot * Plan::kSlotBytes, kVLbo); };
             auto qd = [&](int k) { return make_desc(q_lo + (((k / 4) * Plan::kQHalfBytes + (k % 4) * 32) >> 4)); };
             auto tqd = [&](int k) { return make_desc(tq_lo + (((k / 4) * Plan::kQHalfBytes + (k % 4) * 32) >> 4)); };
-            auto kd = [&](int k) { return make_desc(k_lo + (((k / 4) * 2 * Plan::kKvHalfBytes + (k % 4) * 32) >> 4)); };
+            // B operand of the stacked score MMA: per 64-column half [K (8 KB)][tK (8 KB)]; CTA pair: this CTA's
+            // tensor alone, half after half
+            auto kd = [&](int k) { return make_desc(k_lo + (((k / 4) * (kPair ? 1 : 2) * Plan::kKvHalfBytes + (k % 4) * 32) >> 4)); };
+            // B operand of tQ K^T: the K rows of the same stack; CTA pair: this CTA's 32 rows of K in the slot's second
+            // region (halves of 4 KB)
+            auto k2d = [&](int k) {
+                return kPair ? make_desc(k_lo + ((kHalves * Plan::kKvHalfBytes + (k / 4) * (Plan::kKvHalfBytes / 2) + (k % 4) * 32) >> 4))
+                             : kd(k);
+            };
             auto vd = [&](int k) { return make_desc(v_lo + k * (2048 >> 4)); };
+            // B operand of H~ V: the V atoms of the same slot; CTA pair: this CTA's one atom in the second region
+            auto v2d = [&](int k) { return kPair ? make_desc(v_lo + ((kHalves * Plan::kKvHalfBytes + k * 2048) >> 4)) : vd(k); };
+            // issue and completion tracking in the form the kernel variant needs
+            auto mma_ss0 = [&](uint32_t d, uint64_t a, uint64_t b, uint32_t idesc) {
+                if (kPair) mma_ss_pair<false>(d, a, b, idesc); else mma_ss<false>(d, a, b, idesc);
+            };
+            auto mma_ss1 = [&](uint32_t d, uint64_t a, uint64_t b, uint32_t idesc) {
+                if (kPair) mma_ss_pair<true>(d, a, b, idesc); else mma_ss<true>(d, a, b, idesc);
+            };
+            auto mma_tsx = [&](uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
+                if (kPair) mma_ts_pair(d, a, b, idesc, acc); else mma_ts(d, a, b, idesc, acc);
+            };
+            auto commit = [&](uint32_t bar) { if (kPair) tc_commit_pair(bar); else tc_commit(bar); };
 
             // score MMAs of global tile g (issued by the elected lane), in two parts so that the look-ahead for
             // the next tile can run between them; `last_of_item`: these are the item's last score MMAs
             auto issue_scores_a = [&](int g) {
                 const uint32_t tm_s = tmem + kScoreCol0 + sbuf(g) * kScoreBufStride;
                 TRACE(21, g);         // MMA: about to issue score MMAs
-                mma_ss<false>(tm_s, qd(0), kd(0), kIdescS1);
+                mma_ss0(tm_s, qd(0), kd(0), kIdescS1);
 #pragma unroll
-                for (int k = 1; k < D / 16; ++k) mma_ss<true>(tm_s, qd(k), kd(k), kIdescS1);
+                for (int k = 1; k < D / 16; ++k) mma_ss1(tm_s, qd(k), kd(k), kIdescS1);
+                if (kEarlyS) commit(smem_u32(&bar_s_full[sbuf(g)]));     // S is complete; tS follows
             };
             auto issue_scores_b = [&](int g, int slot, bool last_of_item) {
                 const uint32_t tm_ts = tmem + kScoreCol0 + sbuf(g) * kScoreBufStride + kBlockN;
                 if (kHasTQ) {
-                    if (kHasTKV) mma_ss<true>(tm_ts, tqd(0), kd(0), kIdescS2);
-                    else mma_ss<false>(tm_ts, tqd(0), kd(0), kIdescS2);
+                    if (kHasTKV) mma_ss1(tm_ts, tqd(0), k2d(0), kIdescS2);
+                    else mma_ss0(tm_ts, tqd(0), k2d(0), kIdescS2);
 #pragma unroll
-                    for (int k = 1; k < D / 16; ++k) mma_ss<true>(tm_ts, tqd(k), kd(k), kIdescS2);
+                    for (int k = 1; k < D / 16; ++k) mma_ss1(tm_ts, tqd(k), k2d(k), kIdescS2);
                 }
-                tc_commit(smem_u32(&bar_slot_empty[slot]));
-                tc_commit(smem_u32(&bar_s_full[sbuf(g)]));
-                if (last_of_item) tc_commit(smem_u32(&bar_q_free));
+                commit(smem_u32(&bar_slot_empty[slot]));
+                commit(smem_u32(kEarlyS ? &bar_ts_full[sbuf(g)] : &bar_s_full[sbuf(g)]));
+                if (last_of_item) commit(smem_u32(&bar_q_free));
                 TRACE(2, g);          // MMA: score MMAs of tile g issued
             };
             // value MMAs of tile j of the item (global tile g) out of ring slot `slot`
@@ -799,7 +975,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 TRACE(3, g);          // MMA: about to issue value MMAs
 #pragma unroll
                 for (int k = 0; k < kBlockN / 16; ++k) {
-                    mma_ts(tmem_o, tm_p + k * 8, vd(k), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
+                    mma_tsx(tmem_o, tm_p + k * 8, vd(k), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
                 }
             };
             auto issue_values_h = [&](int j, int g, int slot) {
@@ -807,11 +983,11 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (kHasTQ) {
 #pragma unroll
                     for (int k = 0; k < kBlockN / 16; ++k) {
-                        mma_ts(tmem_t, tm_h + k * 8, vd(k), kIdescHV, (kHasTKV || j > 0 || k > 0) ? 1u : 0u);
+                        mma_tsx(tmem_t, tm_h + k * 8, v2d(k), kIdescHV, (kHasTKV || j > 0 || k > 0) ? 1u : 0u);
                     }
                 }
-                tc_commit(smem_u32(&bar_slot_empty[slot]));
-                tc_commit(smem_u32(&bar_pv_done[g & 1]));
+                commit(smem_u32(&bar_slot_empty[slot]));
+                commit(smem_u32(&bar_pv_done[g & 1]));
                 TRACE(4, g);          // MMA: value MMAs of tile g issued
             };
             // what the burst of global tile g needs: V and K(+2) in shared memory, P~/H~ in tensor memory
@@ -833,7 +1009,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             RingPos pos{0, 0u};
             int g0 = 0;          // global number of the item's first key tile
             int it = 0;
-            for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
+            for (int item = first_item; ok && item < n_items; item += item_stride, ++it) {
                 const Item w = decode(item);
                 const int n_kv = w.n_kv;
                 ok = mbar_wait_warp(smem_u32(&bar_q_full), it & 1, abort_state);
@@ -919,7 +1095,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             }
             if (!ok && leader) {
                 // Abandoning the work: wait (bounded) until the tensor core has drained what was issued.
-                tc_commit(smem_u32(&bar_drain));
+                commit(smem_u32(&bar_drain));
                 const unsigned long long t0 = globaltimer_ns();
                 while (!mbar_try_wait(smem_u32(&bar_drain), 0) && globaltimer_ns() - t0 < 100000000ull) {}
             }
@@ -959,8 +1135,13 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const uint32_t xch_r = xch_m + 3 * kBlockM * 4;                         // partial r
         const uint32_t mbar = smem_u32(&bar_m[quarter]);
         const uint32_t finbar = smem_u32(&bar_fin[quarter]);
+        // arrival on a barrier the MMA-issuing warp waits on: CTA pair -> the first CTA's copy of it
+        auto arrive_at_issuer = [&](uint32_t bar) {
+            if (kPair && !lead_cta) mbar_arrive_cluster(map_to_cta(bar, 0u));
+            else mbar_arrive(bar);
+        };
 
-        for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++it) {
+        for (int item = first_item; ok && item < n_items; item += item_stride, ++it) {
             const Item w = decode(item);
             const int n_kv = w.n_kv;
             float m_ref = -INFINITY;   // running reference max, log2 domain (m of Algorithm 2, lazily updated)
@@ -989,7 +1170,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
                 for (int c0 = 0; c0 < kBlockN; c0 += 32) {
                     TMEM_LD32(tm_s + c0, sv, c0);
-                    if (kHasTQ) TMEM_LD32(tm_ts + c0, tv, c0);
+                    if (kHasTQ && !kEarlyS) TMEM_LD32(tm_ts + c0, tv, c0);
                 }
                 tc_wait_ld();
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
@@ -1039,18 +1220,19 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
                 if (trace_me && quarter == 0 && g < kTraceSteps) g_trace[27][g] = clock64();    // softmax: reference of tile g-1 seen
 #endif
-                if (kHasTQ && j == 0) {
-                    // tO does not change when a per-row constant is subtracted from tS (softmax is shift
-                    // invariant: the constant leaves H~ V - (r/l) O unchanged).  Centring tS on its mean over the
-                    // item's first tile keeps H~ and r small, so that the bf16 rounding of H~ scales with
-                    // |tS - mu| instead of |tS| when the two terms cancel in the epilogue.  (Keys past Lk are
-                    // zero-filled, so their tS is exactly 0 and they drop out of the sum.)
+                // tO does not change when a per-row constant is subtracted from tS (softmax is shift invariant:
+                // the constant leaves H~ V - (r/l) O unchanged).  Centring tS on its mean over the item's first
+                // tile keeps H~ and r small, so that the bf16 rounding of H~ scales with |tS - mu| instead of |tS|
+                // when the two terms cancel in the epilogue.  (Keys past Lk are zero-filled, so their tS is exactly
+                // 0 and they drop out of the sum.)
+                auto centre_of_first_tile = [&]() {
                     float sm4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
                     for (int c = 0; c < kBlockN; ++c) sm4[c & 3] += __uint_as_float(tv[c]);
                     const int n_valid = valid < kBlockN ? valid : kBlockN;
-                    ts_shift = sc * ((sm4[0] + sm4[1]) + (sm4[2] + sm4[3])) / static_cast<float>(n_valid);
-                }
+                    return sc * ((sm4[0] + sm4[1]) + (sm4[2] + sm4[3])) / static_cast<float>(n_valid);
+                };
+                if (kHasTQ && !kEarlyS && j == 0) ts_shift = centre_of_first_tile();
 
                 // m_new = max(m, rowmax), applied lazily: the result does not depend on which
                 // reference is used as long as exp() stays in range.
@@ -1126,9 +1308,18 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     tc_wait_st();
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&bar_p_full[bsel]));
+                    if (lane == 0) arrive_at_issuer(smem_u32(&bar_p_full[bsel]));
                 }
                 if (kHasTQ) {
+                    if (kEarlyS) {
+                        // tS follows S: the MMAs of tQ K^T ran while the exponentials above were computed
+                        if (!mbar_wait_warp(smem_u32(&bar_ts_full[bsel]), sphase(g), abort_state)) { ok = false; break; }
+                        tc_fence_after();
+#pragma unroll
+                        for (int c0 = 0; c0 < kBlockN; c0 += 32) TMEM_LD32(tm_ts + c0, tv, c0);
+                        tc_wait_ld();
+                        if (j == 0) ts_shift = centre_of_first_tile();
+                    }
                     // H~ = P~ . tS, r += rowsum(H~)
                     const uint64_t scsc = pack_f32x2(sc, sc);
                     const uint64_t negshift = pack_f32x2(-ts_shift, -ts_shift);
@@ -1157,7 +1348,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(kSplitHandover ? &bar_h_full[bsel] : &bar_p_full[bsel]));
+                if (lane == 0) arrive_at_issuer(smem_u32(kSplitHandover ? &bar_h_full[bsel] : &bar_p_full[bsel]));
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
                 if (trace_me && g < kTraceSteps) g_trace[13 + ((warp - kFirstSoftmaxWarp) & 3)][g] = clock64();    // softmax warp: arrived
 #endif
@@ -1169,7 +1360,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // cuts the keys into chunks stages nothing), or right after its last V tile if it is the CTA's last.
             int stage_slot_o = 0;
             if (kStageSlots > 0) {
-                const bool has_next = n_items - item > static_cast<int>(gridDim.x);
+                const bool has_next = n_items - item > item_stride;
                 const int next_start = (ring_slot + 2 * (n_kv % kSlots) + (it > 0 ? kStageSlots : 0)) % kSlots;
                 stage_slot_o = has_next ? (next_start + min(kBufs, n_kv)) % kSlots : next_start;
                 ring_slot = next_start;
@@ -1177,9 +1368,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
             if (kGroups == 2 && !finisher) {
                 // This group's share of l and r goes to the group that finishes the item; the exchange words are
-                // single, so the finisher of the item before must have read its own first (it arrives on
-                // `acc_free` after that; at this point that barrier is in the phase of item it - 1 or it).
-                if (it > 0 && !mbar_wait_warp(smem_u32(&bar_acc_free), (it - 1) & 1, abort_state)) { ok = false; break; }
+                // single, so the finisher of the item before must have read its own first.
+                if (it > 0 && !mbar_wait_warp(smem_u32(&bar_fin_read[quarter]), (it - 1) & 1, abort_state)) { ok = false; break; }
                 st_shared_f32(xch_l, l_run);
                 st_shared_f32(xch_r, r_run);
                 __syncwarp();
@@ -1199,6 +1389,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const float f = ex2f(m_other - m_ref);
                     l_run = fmaf(ld_shared_f32(xch_l), f, l_run);
                     r_run = fmaf(ld_shared_f32(xch_r), f, r_run);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&bar_fin_read[quarter]));
                 }
             }
             if (!ok) break;
@@ -1239,7 +1431,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     // O and T are in registers: the next item's first value MMA may overwrite them
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&bar_acc_free));
+                    if (lane == 0) arrive_at_issuer(smem_u32(&bar_acc_free));
                 }
                 if (kSplit) {
 #pragma unroll
@@ -1309,14 +1501,17 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
 
     // Teardown: every role falls through to here (all waits are bounded).
+    // (CTA pair: neither CTA may leave, or free its tensor memory, while the other can still reach into it -- the
+    // first CTA's MMAs read and write both, the second CTA's warps arrive on the first one's barriers.)
     tc_fence_before();
-    __syncthreads();
+    if (kPair) cluster_sync_all(); else __syncthreads();
 #ifdef ATTN_JVP_TRACE
     if (trace_on && threadIdx.x == 0) g_trace[kTraceEvents - 1][1] = clock64();      // CTA ends
 #endif
     if (warp == kMmaWarp) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+        if (kPair) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
 }
 

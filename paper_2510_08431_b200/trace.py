@@ -6,7 +6,7 @@ warp issued the score and value MMAs and when the softmax warps saw the scores, 
 stored P~ and handed the tile back -- plus the mean tile period.  The cycle figures quoted in the design doc and
 profiles/ come from this tool:
 
-    python -m paper_2510_08431_b200.trace --B 1 --H 8 --Lq 18944 --Lk 4096 --D 128 [--mode jvp|kv_free|fwd] [--groups 1|2]
+    python -m paper_2510_08431_b200.trace --B 1 --H 8 --Lq 18944 --Lk 4096 --D 128 [--mode jvp|kv_free|fwd] [--groups 1|2] [--pair 1|2]
 """
 from __future__ import annotations
 
@@ -36,13 +36,14 @@ def build_trace_library() -> str:
     return TRACE_LIB
 
 
-def run(B, H, Lq, Lk, D, mode="jvp", groups=0, first=20, count=6, seed=4):
+def run(B, H, Lq, Lk, D, mode="jvp", groups=0, first=20, count=6, seed=4, pair=0):
     """Runs the shape three times through the trace build and returns the [EVENTS][STEPS] stamp array."""
     lib = ctypes.CDLL(build_trace_library())
     x = synth.make_inputs(B, H, Lq, Lk, D, 1.0, 0.5, seed, kv_tangent_free=(mode != "jvp"))
     g = {k: (None if t is None else t.cuda()) for k, t in x.items()}
     flags = {"jvp": 0, "kv_free": binding.KV_TANGENT_FREE, "fwd": binding.FWD_ONLY}[mode]
     lib.attn_jvp_set_tuning(binding.TUNE_SOFTMAX_GROUPS, int(groups))
+    lib.attn_jvp_set_tuning(binding.TUNE_CTA_PAIR, int(pair))
     o = torch.empty_like(g["q"]); to = torch.empty_like(g["q"])
     lse = torch.empty((B, H, Lq), dtype=torch.float32, device="cuda")
     vp = ctypes.c_void_p
@@ -91,9 +92,10 @@ def main():
     ap.add_argument("--D", type=int, default=128)
     ap.add_argument("--mode", default="jvp", choices=["jvp", "kv_free", "fwd"])
     ap.add_argument("--groups", type=int, default=0)
+    ap.add_argument("--pair", type=int, default=0, help="CTA-pair kernel: 0 library's choice, 1 off, 2 on")
     ap.add_argument("--first", type=int, default=20); ap.add_argument("--count", type=int, default=4)
     a = ap.parse_args()
-    report(run(a.B, a.H, a.Lq, a.Lk, a.D, a.mode, a.groups), a.first, a.count)
+    report(run(a.B, a.H, a.Lq, a.Lk, a.D, a.mode, a.groups, pair=a.pair), a.first, a.count)
 
 
 if __name__ == "__main__":
