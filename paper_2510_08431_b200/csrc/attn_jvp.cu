@@ -40,7 +40,7 @@ struct DeviceState {
     std::atomic<int*> host_status_dev{nullptr};   // ... and its device-side address (published first)
     std::atomic<bool> unwatched_launch{false};    // a kernel ran here before the status word existed
     std::atomic<int> dyn_smem[2][3][2][2];        // dynamic shared memory per kernel instantiation, 0 = not set up
-    std::atomic<int> dyn_smem_pair[2];            // ... of the CTA-pair kernels
+    std::atomic<int> dyn_smem_pair[3][2];         // ... of the CTA-pair kernels
     std::atomic<void*> static_scratch{nullptr};   // device address of the built-in scratch array
 };
 DeviceState g_dev[kMaxDevices];
@@ -51,22 +51,28 @@ std::atomic<EncodeTiledFn> g_encode_tiled{nullptr};
 std::atomic<int> g_tune_softmax_groups{0};
 std::atomic<int> g_tune_cta_pair{0};
 
-// Softmax groups of the CTA-pair kernel (measured: one group is 3-8 % faster than two there as well).
-int softmax_groups_for_pair() {
+// Softmax groups of the CTA-pair kernel (measured: with tangents one group is 3-8 % faster than two there as well;
+// the forward-only pair is 14 % faster with two).
+int softmax_groups_for_pair(int mode) {
     const int forced = g_tune_softmax_groups.load(std::memory_order_relaxed);
-    return forced == 2 ? 2 : 1;
+    if (forced == 1 || forced == 2) return forced;
+    return mode == attn_jvp::kModeFwdOnly ? 2 : 1;
 }
 
 // Whether a call runs on the CTA-pair kernel (clusters of two CTAs sharing the K/V operand tiles and one MMA
 // instruction stream).  It exists for the full JVP at D = 128.
 bool use_cta_pair(int mode, int D, bool split, int tiles_per_item) {
-    if (mode != attn_jvp::kModeJvp || D != 128 || split) return false;
+    if (D != 128 || split) return false;
     const int forced = g_tune_cta_pair.load(std::memory_order_relaxed);
     if (forced == 1) return false;
     if (forced == 2) return true;
-    // Measured on B200: 4-20 % faster than one CTA per query tile from about eight key tiles per item on (12 % on
-    // the 32760-token self-attention workloads), 4 % slower with two key tiles per item.
-    return tiles_per_item >= 6;
+    // Measured on B200.  Full JVP: 4-20 % faster than one CTA per query tile from about eight key tiles per item on
+    // (12 % on the 32760-token self-attention workloads), 4 % slower with two key tiles per item.  Forward only:
+    // 7-9 % faster (with two softmax groups) on the image- and video-length workloads, slower on short items.
+    // Tangent-free K/V: 3-6 % slower everywhere, so it stays on one CTA per query tile.
+    if (mode == attn_jvp::kModeJvp) return tiles_per_item >= 6;
+    if (mode == attn_jvp::kModeFwdOnly) return tiles_per_item >= 32;
+    return false;
 }
 
 // Softmax warpgroups per CTA for a kernel variant: two groups take alternate key tiles, which pays where the
@@ -175,7 +181,7 @@ template <int D, int MODE, bool SPLIT, int GROUPS, bool PAIR = false>
 int launch(const CUtensorMap* maps, const KernelArgs& ka, dim3 grid, cudaStream_t stream, DeviceState& st) {
     auto kern = attn_jvp::attn_jvp_fwd_kernel<D, MODE, SPLIT, GROUPS, PAIR>;
     using Plan = attn_jvp::SmemPlan<D, GROUPS>;
-    std::atomic<int>& slot = PAIR ? st.dyn_smem_pair[GROUPS - 1] : st.dyn_smem[D == 128][MODE][SPLIT][GROUPS - 1];
+    std::atomic<int>& slot = PAIR ? st.dyn_smem_pair[MODE][GROUPS - 1] : st.dyn_smem[D == 128][MODE][SPLIT][GROUPS - 1];
     int smem = slot.load(std::memory_order_acquire);
     if (smem == 0) {
         // dynamic shared memory = the operand layout (declared 1024-byte aligned in the kernel) plus the exchange
@@ -364,8 +370,18 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
         const long long max_pairs = st.sm_count / 2;
         const long long n_pairs = (persistent && n_pair_items > max_pairs) ? max_pairs : n_pair_items;
         const dim3 pair_grid((unsigned)(2 * n_pairs), 1, 1);
-        if (softmax_groups_for_pair() == 2) return launch<128, attn_jvp::kModeJvp, false, 2, true>(maps, ka, pair_grid, stream, st);
-        return launch<128, attn_jvp::kModeJvp, false, 1, true>(maps, ka, pair_grid, stream, st);
+        const bool two = softmax_groups_for_pair(mode) == 2;
+        switch (mode) {
+            case attn_jvp::kModeJvp:
+                return two ? launch<128, attn_jvp::kModeJvp, false, 2, true>(maps, ka, pair_grid, stream, st)
+                           : launch<128, attn_jvp::kModeJvp, false, 1, true>(maps, ka, pair_grid, stream, st);
+            case attn_jvp::kModeKvTangentFree:
+                return two ? launch<128, attn_jvp::kModeKvTangentFree, false, 2, true>(maps, ka, pair_grid, stream, st)
+                           : launch<128, attn_jvp::kModeKvTangentFree, false, 1, true>(maps, ka, pair_grid, stream, st);
+            default:
+                return two ? launch<128, attn_jvp::kModeFwdOnly, false, 2, true>(maps, ka, pair_grid, stream, st)
+                           : launch<128, attn_jvp::kModeFwdOnly, false, 1, true>(maps, ka, pair_grid, stream, st);
+        }
     }
     const long long n_ctas = (persistent && n_items > st.sm_count) ? st.sm_count : n_items;
     const dim3 grid((unsigned)n_ctas, 1, 1);

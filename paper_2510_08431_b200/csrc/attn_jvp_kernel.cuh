@@ -472,7 +472,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const __grid_constant__ CUtensorMap tm_tk, const __grid_constant__ CUtensorMap tm_tv,
                     const __grid_constant__ CUtensorMap tm_o, const __grid_constant__ CUtensorMap tm_to,
                     const __grid_constant__ CUtensorMap tm_k32, const KernelArgs args) {
-    static_assert(!kPair || (MODE == kModeJvp && D == 128 && !kSplit), "the CTA-pair variant exists for the full JVP at D = 128");
+    static_assert(!kPair || (D == 128 && !kSplit), "the CTA-pair variant exists at D = 128, without key chunks");
     using Plan = SmemPlan<D, kGroups>;
     constexpr int kFirstSoftmaxWarp = first_softmax_warp(kGroups);
     constexpr int kHalves = Plan::kHalves;
@@ -716,16 +716,19 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 uint32_t dst, bar;
                 if (!acquire(slot, dst, bar)) return false;
                 if (kPair) {
-                    // The stacked operand [K ; tK] is split by tensor: this CTA holds K (first CTA) or tK (second) as
-                    // [half 0 (8 KB)][half 1 (8 KB)].  The N = 64 operand of tQ K^T is split by rows: K rows
-                    // 32 r .. 32 r + 31 as [half 0 (4 KB)][half 1 (4 KB)] in the slot's second region.
-                    constexpr uint32_t kTxPerCta = 2 * Plan::kKvHalfBytes + Plan::kKvHalfBytes;     // 16 KB + 8 KB
+                    // With K/V tangents the stacked operand [K ; tK] is split by tensor: this CTA holds K (first CTA)
+                    // or tK (second) as [half 0 (8 KB)][half 1 (8 KB)], and the N = 64 operand of tQ K^T is split by
+                    // rows: K rows 32 r .. 32 r + 31 as [half 0 (4 KB)][half 1 (4 KB)] in the slot's second region.
+                    // Without them every score MMA has N = 64 and takes that row split alone, from the slot's start.
+                    constexpr uint32_t kTxPerCta = (kHasTKV ? 2 * Plan::kKvHalfBytes : 0) + Plan::kKvHalfBytes;
+                    constexpr uint32_t kRows32Off = kHasTKV ? kPairRegionB : 0;
                     if (lead_cta) mbar_arrive_expect_tx(smem_u32(&bar_slot_full[slot]), 2 * kTxPerCta);
                     const int row0 = (w.tile0 + j) * kBlockN;
 #pragma unroll
                     for (int hf = 0; hf < kHalves; ++hf) {
-                        tma_load_4d_pair(dst + hf * Plan::kKvHalfBytes, lead_cta ? &tm_k : &tm_tk, bar, hf * 64, w.h, row0, w.b);
-                        tma_load_4d_pair(dst + kPairRegionB + hf * (Plan::kKvHalfBytes / 2), &tm_k32, bar, hf * 64, w.h,
+                        if (kHasTKV)
+                            tma_load_4d_pair(dst + hf * Plan::kKvHalfBytes, lead_cta ? &tm_k : &tm_tk, bar, hf * 64, w.h, row0, w.b);
+                        tma_load_4d_pair(dst + kRows32Off + hf * (Plan::kKvHalfBytes / 2), &tm_k32, bar, hf * 64, w.h,
                                          row0 + 32 * static_cast<int>(cta_rank), w.b);
                     }
                     return true;
@@ -745,15 +748,19 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 uint32_t dst, bar;
                 if (!acquire(slot, dst, bar)) return false;
                 if (kPair) {
-                    // [V | tV] is split by tensor: this CTA holds V (first CTA) or tV (second) as two 64-wide N atoms.
-                    // The N = 128 operand of H~ V is split by columns: V atom r in the slot's second region.
-                    constexpr uint32_t kTxPerCta = 2 * Plan::kKvHalfBytes + Plan::kKvHalfBytes;
+                    // With K/V tangents [V | tV] is split by tensor: this CTA holds V (first CTA) or tV (second) as two
+                    // 64-wide N atoms, and the N = 128 operand of H~ V is split by columns: V atom r in the slot's
+                    // second region.  Without them every value MMA has N = 128 and takes that column split alone.
+                    constexpr uint32_t kTxPerCta = (kHasTKV ? 2 * Plan::kKvHalfBytes : 0) + Plan::kKvHalfBytes;
+                    constexpr uint32_t kAtomOff = kHasTKV ? kPairRegionB : 0;
                     if (lead_cta) mbar_arrive_expect_tx(smem_u32(&bar_slot_full[slot]), 2 * kTxPerCta);
                     const int row0 = (w.tile0 + j) * kBlockN;
+                    if (kHasTKV) {
 #pragma unroll
-                    for (int hf = 0; hf < kHalves; ++hf)
-                        tma_load_4d_pair(dst + hf * Plan::kKvHalfBytes, lead_cta ? &tm_v : &tm_tv, bar, hf * 64, w.h, row0, w.b);
-                    tma_load_4d_pair(dst + kPairRegionB, &tm_v, bar, 64 * static_cast<int>(cta_rank), w.h, row0, w.b);
+                        for (int hf = 0; hf < kHalves; ++hf)
+                            tma_load_4d_pair(dst + hf * Plan::kKvHalfBytes, lead_cta ? &tm_v : &tm_tv, bar, hf * 64, w.h, row0, w.b);
+                    }
+                    tma_load_4d_pair(dst + kAtomOff, &tm_v, bar, 64 * static_cast<int>(cta_rank), w.h, row0, w.b);
                     return true;
                 }
                 mbar_arrive_expect_tx(bar, kVTx);
@@ -818,7 +825,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
                     for (int hf = 0; hf < kHalves; ++hf) {
                         tma_load_4d_pair(smem_q + hf * Plan::kQHalfBytes, &tm_q, qbar, hf * 64, w.h, w.q0, w.b);
-                        tma_load_4d_pair(smem_tq + hf * Plan::kQHalfBytes, &tm_tq, qbar, hf * 64, w.h, w.q0, w.b);
+                        if (kHasTQ) tma_load_4d_pair(smem_tq + hf * Plan::kQHalfBytes, &tm_tq, qbar, hf * 64, w.h, w.q0, w.b);
                     }
                 } else {
                     mbar_arrive_expect_tx(qbar, kQTx);
@@ -922,16 +929,20 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             auto tqd = [&](int k) { return make_desc(tq_lo + (((k / 4) * Plan::kQHalfBytes + (k % 4) * 32) >> 4)); };
             // B operand of the stacked score MMA: per 64-column half [K (8 KB)][tK (8 KB)]; CTA pair: this CTA's
             // tensor alone, half after half
-            auto kd = [&](int k) { return make_desc(k_lo + (((k / 4) * (kPair ? 1 : 2) * Plan::kKvHalfBytes + (k % 4) * 32) >> 4)); };
-            // B operand of tQ K^T: the K rows of the same stack; CTA pair: this CTA's 32 rows of K in the slot's second
-            // region (halves of 4 KB)
+            // CTA pair without K/V tangents: this CTA's 32 rows of K, halves of 4 KB from the slot's start (see load_k)
+            constexpr bool kPairRowsOnly = kPair && !kHasTKV;
+            constexpr uint32_t kPairOff2 = kHasTKV ? kHalves * Plan::kKvHalfBytes : 0;   // pair: the slot's second region
+            auto kd = [&](int k) {
+                return make_desc(k_lo + (((k / 4) * (kPairRowsOnly ? Plan::kKvHalfBytes / 2 : (kPair ? 1 : 2) * Plan::kKvHalfBytes)
+                                          + (k % 4) * 32) >> 4));
+            };
+            // B operand of tQ K^T: the K rows of the same stack; CTA pair: this CTA's 32 rows of K (halves of 4 KB)
             auto k2d = [&](int k) {
-                return kPair ? make_desc(k_lo + ((kHalves * Plan::kKvHalfBytes + (k / 4) * (Plan::kKvHalfBytes / 2) + (k % 4) * 32) >> 4))
-                             : kd(k);
+                return kPair ? make_desc(k_lo + ((kPairOff2 + (k / 4) * (Plan::kKvHalfBytes / 2) + (k % 4) * 32) >> 4)) : kd(k);
             };
             auto vd = [&](int k) { return make_desc(v_lo + k * (2048 >> 4)); };
-            // B operand of H~ V: the V atoms of the same slot; CTA pair: this CTA's one atom in the second region
-            auto v2d = [&](int k) { return kPair ? make_desc(v_lo + ((kHalves * Plan::kKvHalfBytes + k * 2048) >> 4)) : vd(k); };
+            // B operand of H~ V: the V atoms of the same slot; CTA pair: this CTA's one atom of V
+            auto v2d = [&](int k) { return kPair ? make_desc(v_lo + ((kPairOff2 + k * 2048) >> 4)) : vd(k); };
             // issue and completion tracking in the form the kernel variant needs
             auto mma_ss0 = [&](uint32_t d, uint64_t a, uint64_t b, uint32_t idesc) {
                 if (kPair) mma_ss_pair<false>(d, a, b, idesc); else mma_ss<false>(d, a, b, idesc);
@@ -1379,9 +1390,14 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             }
 
             // Epilogue: O/l, L = m + log l, tO = (T - r (O/l)) / l, once the item's last value MMAs are complete
-            // (which implies all earlier ones)
+            // (which implies all earlier ones).  A parity wait on bar_pv_done[g & 1] for tile g means what it should
+            // only once the value MMAs of tile g - 2 (the barrier's previous phase) are known to be complete.  The
+            // scores of tile g_last have been seen, and their completion implies that of everything issued before
+            // them: the value MMAs up to tile g_last - kBufs, and for an item's leading tiles those of all earlier
+            // items.  That covers g_last - 3, so tile g_last - 1 can be waited for first, and g_last after it.
             const int g_last = g0 + n_kv - 1;
-            ok = mbar_wait_warp(smem_u32(&bar_pv_done[g_last & 1]), (g_last >> 1) & 1, abort_state);
+            if (n_kv >= 2) ok = mbar_wait_warp(smem_u32(&bar_pv_done[(g_last - 1) & 1]), ((g_last - 1) >> 1) & 1, abort_state);
+            if (ok) ok = mbar_wait_warp(smem_u32(&bar_pv_done[g_last & 1]), (g_last >> 1) & 1, abort_state);
             if (ok && kGroups == 2) {
                 // the other group's sums, brought to the final reference (it last knew m_other; 0 if it had no tile)
                 ok = mbar_wait_warp(finbar, it & 1, abort_state);
