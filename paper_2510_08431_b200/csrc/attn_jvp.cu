@@ -180,7 +180,7 @@ bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
 template <int D, int MODE, bool SPLIT, int GROUPS, bool PAIR = false>
 int launch(const CUtensorMap* maps, const KernelArgs& ka, dim3 grid, cudaStream_t stream, DeviceState& st) {
     auto kern = attn_jvp::attn_jvp_fwd_kernel<D, MODE, SPLIT, GROUPS, PAIR>;
-    using Plan = attn_jvp::SmemPlan<D, GROUPS>;
+    using Plan = attn_jvp::SmemPlan<D, MODE, GROUPS, PAIR>;
     std::atomic<int>& slot = PAIR ? st.dyn_smem_pair[MODE][GROUPS - 1] : st.dyn_smem[D == 128][MODE][SPLIT][GROUPS - 1];
     int smem = slot.load(std::memory_order_acquire);
     if (smem == 0) {

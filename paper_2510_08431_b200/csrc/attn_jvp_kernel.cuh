@@ -107,15 +107,27 @@ struct KernelArgs {
     int n_items;        // work items = n_q_tiles * H * B * splits; the grid's CTAs share them round-robin
 };
 
-template <int D, int kGroups = 1>
+// Shared-memory plan of a kernel variant.
+//   One Q/tQ buffer (full JVP at D = 128, and every CTA-pair variant): Q, tQ resident, ring slots of one primal +
+//   one tangent tile (= one 128 x D bf16 output tile, which is what the ring's staging slots rely on).
+//   Two Q/tQ buffers (the variants that leave room: no K/V tangents, or D = 64): the next item's Q, tQ are loaded
+//   while the current item runs, ring slots hold exactly what the mode loads, and an item's output tiles are staged
+//   in its own Q/tQ buffer (dead once its last value MMAs are complete) instead of in ring slots.
+template <int D, int MODE, int kGroups, bool kPair>
 struct SmemPlan {
     static constexpr int kHalves = D / 64;                 // 64-element (128-byte) swizzle atoms per row
     static constexpr int kQHalfBytes = kBlockM * 128;      // 16 KB: 128 rows x 128 B
     static constexpr int kQBytes = kHalves * kQHalfBytes;
     static constexpr int kKvHalfBytes = kBlockN * 128;     // 8 KB: 64 rows x 128 B
-    static constexpr int kSlotBytes = 2 * kHalves * kKvHalfBytes;  // primal + tangent tile
-    static constexpr int kSlots = (D == 128) ? 5 : 8;
-    static constexpr int kOperandBytes = 2 * kQBytes + kSlots * kSlotBytes;
+    static constexpr bool kDoubleQ = !kPair && (MODE != kModeJvp || D == 64);
+    static constexpr int kQSets = kDoubleQ ? 2 : 1;
+    static constexpr int kQSetBytes = (kDoubleQ && MODE == kModeFwdOnly) ? kQBytes : 2 * kQBytes;   // Q (+ tQ)
+    static constexpr int kTilesPerSlot = (!kDoubleQ || MODE == kModeJvp) ? 2 : 1;                   // primal (+ tangent)
+    static constexpr int kSlotBytes = kTilesPerSlot * kHalves * kKvHalfBytes;
+    static constexpr int kRoom = 224 * 1024 - kQSets * kQSetBytes;
+    static constexpr int kSlots = kDoubleQ ? (kRoom / kSlotBytes < 8 ? kRoom / kSlotBytes : 8) : ((D == 128) ? 5 : 8);
+    static constexpr int kRingOffset = kQSets * kQSetBytes;
+    static constexpr int kOperandBytes = kRingOffset + kSlots * kSlotBytes;
     // Two softmax groups exchange four per-row fp32 values through shared memory (reference max, centring
     // constant of tS, partial l and r), placed after the operand tiles.
     static constexpr int kExchangeBytes = (kGroups == 2) ? 4 * kBlockM * 4 : 0;
@@ -473,7 +485,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const __grid_constant__ CUtensorMap tm_o, const __grid_constant__ CUtensorMap tm_to,
                     const __grid_constant__ CUtensorMap tm_k32, const KernelArgs args) {
     static_assert(!kPair || (D == 128 && !kSplit), "the CTA-pair variant exists at D = 128, without key chunks");
-    using Plan = SmemPlan<D, kGroups>;
+    using Plan = SmemPlan<D, MODE, kGroups, kPair>;
+    constexpr bool kDoubleQ = Plan::kDoubleQ;
     constexpr int kFirstSoftmaxWarp = first_softmax_warp(kGroups);
     constexpr int kHalves = Plan::kHalves;
     constexpr int kSlots = Plan::kSlots;
@@ -482,7 +495,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // The bf16 output tiles leave through shared memory and TMA stores: at the end of every item the ring gives
     // up one slot per output tensor (a slot is exactly one 128 x D bf16 tile).  The split-KV kernel writes its
     // fp32 partial results straight from registers and stages nothing.
-    constexpr int kStageSlots = kSplit ? 0 : (kHasTQ ? 2 : 1);
+    constexpr int kStageSlots = kSplit ? 0 : (kHasTQ ? 2 : 1);       // output tiles staged per item ...
+    constexpr int kRingStage = kDoubleQ ? 0 : kStageSlots;           // ... of which in ring slots (else in the item's Q/tQ buffer)
     // With tK = tV = 0 the tensor pipe has spare time and a key tile takes as long as the chain softmax -> value
     // MMAs -> score MMAs: there P~ is handed to the MMA warp as soon as it is stored, and the MMAs that read it run
     // beside the H~ arithmetic (H~ follows through a barrier of its own).  In the full mode the MMA warp never
@@ -501,10 +515,10 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     constexpr int kScoreCol0 = (kBufs == 3) ? 128 : 256;     // first column of score buffer 0
     static_assert(kScoreCol0 + kBufs * kScoreBufStride <= kTmemCols, "score buffers must fit into tensor memory");
     static_assert((kHasTQ ? 2 * D : D) <= kScoreCol0, "accumulators and score buffers overlap");
-    static_assert(Plan::kSlotBytes == Plan::kQBytes, "an output tile must fill one ring slot");
+    static_assert(kDoubleQ || Plan::kSlotBytes == Plan::kQBytes, "an output tile must fill one ring slot");
 
     extern __shared__ __align__(1024) uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bar_q_full;     // Q, tQ of the current work item are in shared memory
+    __shared__ __align__(8) uint64_t bar_q_full[2];  // Q, tQ of a work item are in shared memory (one barrier per Q/tQ buffer)
     __shared__ __align__(8) uint64_t bar_q_free;     // every score MMA of the item has completed: Q, tQ may be replaced
     __shared__ __align__(8) uint64_t bar_slot_full[kSlots];
     __shared__ __align__(8) uint64_t bar_slot_empty[kSlots];
@@ -539,21 +553,47 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const int first_item = kPair ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
     const int item_stride = kPair ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
     struct Item { int q0, h, b, split, tile0, n_kv; };
-    auto decode = [&](int item) -> Item {
-        Item w;
-        w.q0 = (item % args.n_q_tiles) * (kPair ? 2 * kBlockM : kBlockM) + static_cast<int>(cta_rank) * kBlockM;
+    // Work item number -> (query tile, head, batch [, chunk]).  The roles walk their items with a fixed stride, so
+    // after the first item the three indices are advanced by the stride's own decomposition (carry by compare and
+    // subtract) instead of being divided out again: the divisions would sit on the critical path of every item
+    // hand-over, once per role.
+    struct Walk { int qt, h, z; };
+    auto walk_init = [&](int item) -> Walk {
+        Walk k;
+        k.qt = item % args.n_q_tiles;
         const int rest = item / args.n_q_tiles;
-        w.h = rest % args.H;
-        const int z = rest / args.H;
-        w.b = kSplit ? z / args.splits : z;
-        w.split = kSplit ? z % args.splits : 0;
+        k.h = rest % args.H;
+        k.z = rest / args.H;
+        return k;
+    };
+    const Walk walk_stride = walk_init(item_stride);
+    auto walk_step = [&](Walk& k) {
+        k.qt += walk_stride.qt;
+        if (k.qt >= args.n_q_tiles) { k.qt -= args.n_q_tiles; ++k.h; }
+        k.h += walk_stride.h;
+        if (k.h >= args.H) { k.h -= args.H; ++k.z; }
+        k.z += walk_stride.z;
+    };
+    auto item_of = [&](const Walk& k) -> Item {
+        Item w;
+        w.q0 = k.qt * (kPair ? 2 * kBlockM : kBlockM) + static_cast<int>(cta_rank) * kBlockM;
+        w.h = k.h;
+        w.b = kSplit ? k.z / args.splits : k.z;
+        w.split = kSplit ? k.z % args.splits : 0;
         w.tile0 = kSplit ? w.split * args.tiles_per_split : 0;       // first key tile of this item
         w.n_kv = kSplit ? min(args.tiles_per_split, args.n_kv_tiles - w.tile0) : args.n_kv_tiles;
         return w;
     };
     const int n_items = args.n_items;
-    auto sbuf = [](int g) -> int { return kBufs == 2 ? (g & 1) : g % kBufs; };
-    auto sphase = [](int g) -> uint32_t { return static_cast<uint32_t>(kBufs == 2 ? (g >> 1) : g / kBufs) & 1u; };
+    // Two Q/tQ buffers, no key chunks (every item then has the same number of key tiles): the key tiles of all of a
+    // CTA's items form one stream.  The score MMAs of an item's leading tiles are issued in the last bursts of the
+    // item before (its Q, tQ are resident by then), and the ring carries their K tiles in that order, so that an
+    // item boundary costs the MMA warp and the producer nothing.
+    const bool stream_items = kDoubleQ && !kSplit && args.n_kv_tiles >= kBufs;
+    // Score buffer and barrier phase of a key tile, g % kBufs and (g / kBufs) & 1, carried along tile by tile (a
+    // division by three per use would sit on the MMA warp's critical chain of dependent instructions).
+    struct BufPos { int buf; uint32_t phase; };
+    auto next_buf = [](BufPos& p) { if (++p.buf == kBufs) { p.buf = 0; p.phase ^= 1u; } };
 
     // An earlier CTA of this (or a previous) launch gave up: do not start.  One thread reads
     // the flag so that the whole CTA takes the same decision.
@@ -568,9 +608,12 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     if (trace_on && threadIdx.x == 0) g_trace[kTraceEvents - 1][0] = clock64();      // CTA begins
 #endif
     const uint32_t smem_base = smem_u32(smem_raw);
-    const uint32_t smem_q = smem_base;
-    const uint32_t smem_tq = smem_base + Plan::kQBytes;
-    const uint32_t smem_ring = smem_base + 2 * Plan::kQBytes;
+    // Q/tQ buffer of item number `it`, its `full` barrier and that barrier's phase
+    auto q_addr = [&](int it) -> uint32_t { return smem_base + (kDoubleQ ? (it & 1) * Plan::kQSetBytes : 0); };
+    auto tq_addr = [&](int it) -> uint32_t { return q_addr(it) + Plan::kQBytes; };
+    auto q_full_bar = [&](int it) -> uint32_t { return smem_u32(&bar_q_full[kDoubleQ ? (it & 1) : 0]); };
+    auto q_full_phase = [](int it) -> uint32_t { return static_cast<uint32_t>(kDoubleQ ? (it >> 1) : it) & 1u; };
+    const uint32_t smem_ring = smem_base + Plan::kRingOffset;
 
     AbortState abort_state{&cta_abort, args.host_status};
 
@@ -587,7 +630,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     }
 
     if (threadIdx.x == 0) {
-        mbar_init(smem_u32(&bar_q_full), 1);
+        mbar_init(smem_u32(&bar_q_full[0]), 1);
+        mbar_init(smem_u32(&bar_q_full[1]), 1);
         mbar_init(smem_u32(&bar_q_free), 1);
         for (int i = 0; i < kSlots; ++i) {
             mbar_init(smem_u32(&bar_slot_full[i]), 1);
@@ -614,7 +658,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 #ifdef ATTN_JVP_DEBUG
         if (blockIdx.x == 0) {
-            const void* named[] = {&bar_q_full, &bar_q_free, &bar_slot_full[0], &bar_slot_empty[0], &bar_s_full[0],
+            const void* named[] = {&bar_q_full[0], &bar_q_free, &bar_slot_full[0], &bar_slot_empty[0], &bar_s_full[0],
                                    &bar_p_full[0], &bar_h_full[0], &bar_pv_done[0], &bar_acc_free, &bar_drain,
                                    &bar_stage_ready, &bar_stage_full, &bar_m[0], &bar_fin[0]};
             for (int i = 0; i < 14; ++i) g_barrier_layout[i] = smem_u32(named[i]);
@@ -687,7 +731,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             constexpr uint32_t kVTx = kKTx;
             // CTA pair: the `full` barriers that count, the MMA-issuing warp's, are the first CTA's; both CTAs' loads
             // report their bytes there and the first CTA's producer announces the bytes of both.
-            const uint32_t qbar = kPair ? map_to_cta(smem_u32(&bar_q_full), 0u) : smem_u32(&bar_q_full);
+            // bytes between the 64-column halves of a K slot: the tangent tile's half sits between them unless the
+            // slot holds the primal tile alone (two Q/tQ buffers, no K/V tangents)
+            constexpr uint32_t kKHalfStride = Plan::kTilesPerSlot * Plan::kKvHalfBytes;
             // pair: offset of the second operand region of a ring slot (the halves of K / V that the N = 64 and
             // N = 128 MMAs take from each CTA at a common offset)
             constexpr uint32_t kPairRegionB = kHalves * Plan::kKvHalfBytes;   // 16 KB at D = 128
@@ -737,9 +783,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 // per 64-column half: [K_half (8 KB)][tK_half (8 KB)] so that [K ; tK] is one N = 128 operand
 #pragma unroll
                 for (int hf = 0; hf < kHalves; ++hf) {
-                    tma_load_4d(dst + hf * 2 * Plan::kKvHalfBytes, &tm_k, bar, hf * 64, w.h, (w.tile0 + j) * kBlockN, w.b);
+                    tma_load_4d(dst + hf * kKHalfStride, &tm_k, bar, hf * 64, w.h, (w.tile0 + j) * kBlockN, w.b);
                     if (kHasTKV)
-                        tma_load_4d(dst + hf * 2 * Plan::kKvHalfBytes + Plan::kKvHalfBytes, &tm_tk, bar, hf * 64, w.h, (w.tile0 + j) * kBlockN, w.b);
+                        tma_load_4d(dst + hf * kKHalfStride + Plan::kKvHalfBytes, &tm_tk, bar, hf * 64, w.h, (w.tile0 + j) * kBlockN, w.b);
                 }
                 return true;
             };
@@ -781,19 +827,20 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             auto store_staged = [&]() -> bool {
                 if (!mbar_wait(smem_u32(&bar_stage_full), stage_it & 1, abort_state)) return false;
                 TRACE(17, stage_it);  // producer: staged tiles complete, stores issued next
+                // staged in two ring slots, or (two Q/tQ buffers) in the item's own Q and tQ buffer
+                const uint32_t src_o = kDoubleQ ? q_addr(stage_it) : smem_ring + stage_slot[0] * Plan::kSlotBytes;
+                const uint32_t src_t = kDoubleQ ? tq_addr(stage_it) : smem_ring + stage_slot[1] * Plan::kSlotBytes;
 #pragma unroll
                 for (int hf = 0; hf < kHalves; ++hf) {
                     if (kPair && stage_w.q0 >= args.Lq) break;     // second CTA of a pair whose rows all lie past Lq
-                    tma_store_4d(&tm_o, smem_ring + stage_slot[0] * Plan::kSlotBytes + hf * Plan::kQHalfBytes,
-                                 hf * 64, stage_w.h, stage_w.q0, stage_w.b);
+                    tma_store_4d(&tm_o, src_o + hf * Plan::kQHalfBytes, hf * 64, stage_w.h, stage_w.q0, stage_w.b);
                     if (kStageSlots > 1)
-                        tma_store_4d(&tm_to, smem_ring + stage_slot[1] * Plan::kSlotBytes + hf * Plan::kQHalfBytes,
-                                     hf * 64, stage_w.h, stage_w.q0, stage_w.b);
+                        tma_store_4d(&tm_to, src_t + hf * Plan::kQHalfBytes, hf * 64, stage_w.h, stage_w.q0, stage_w.b);
                 }
                 tma_store_commit();
                 tma_store_wait_read();
                 // the slots go back to the ring (their `empty` phase is completed here instead of by an MMA commit)
-                for (int s = 0; s < kStageSlots; ++s) mbar_arrive(smem_u32(&bar_slot_empty[stage_slot[s]]));
+                for (int s = 0; s < kRingStage; ++s) mbar_arrive(smem_u32(&bar_slot_empty[stage_slot[s]]));
                 TRACE(18, stage_it);  // producer: staging slots back in the ring
                 stage_pending = false;
                 return true;
@@ -801,7 +848,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // hands the staging slots of item number `of_it` to the softmax warps; nothing is loaded into them, so
             // their `full` phase is completed by a plain arrival to keep the ring's parities in step
             auto acquire_stage = [&](int of_it, const Item& of_w) -> bool {
-                for (int s = 0; s < kStageSlots; ++s) {
+                for (int s = 0; s < kRingStage; ++s) {
                     uint32_t dst, bar;
                     if (!acquire(stage_slot[s], dst, bar)) return false;
                     if (!kPair || lead_cta) mbar_arrive(smem_u32(&bar_slot_full[stage_slot[s]]));
@@ -813,59 +860,102 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 stage_w = of_w;
                 return true;
             };
-            Item prev_w{};
-            int it = 0;
-            for (int item = first_item; ok && item < n_items; item += item_stride, ++it) {
-                w = decode(item);
-                if (it > 0) ok = mbar_wait(smem_u32(&bar_q_free), (it - 1) & 1, abort_state);
-                if (!ok) break;
-                TRACE(1, it);         // producer: Q, tQ may be replaced
+            // Q, tQ of item number `n` (work item `wi`) into its buffer
+            auto load_q = [&](int n, const Item& wi) {
+                const uint32_t dq = q_addr(n), dtq = tq_addr(n);
                 if (kPair) {
-                    if (lead_cta) mbar_arrive_expect_tx(smem_u32(&bar_q_full), 2 * kQTx);
+                    const uint32_t qbar = map_to_cta(q_full_bar(n), 0u);
+                    if (lead_cta) mbar_arrive_expect_tx(q_full_bar(n), 2 * kQTx);
 #pragma unroll
                     for (int hf = 0; hf < kHalves; ++hf) {
-                        tma_load_4d_pair(smem_q + hf * Plan::kQHalfBytes, &tm_q, qbar, hf * 64, w.h, w.q0, w.b);
-                        if (kHasTQ) tma_load_4d_pair(smem_tq + hf * Plan::kQHalfBytes, &tm_tq, qbar, hf * 64, w.h, w.q0, w.b);
+                        tma_load_4d_pair(dq + hf * Plan::kQHalfBytes, &tm_q, qbar, hf * 64, wi.h, wi.q0, wi.b);
+                        if (kHasTQ) tma_load_4d_pair(dtq + hf * Plan::kQHalfBytes, &tm_tq, qbar, hf * 64, wi.h, wi.q0, wi.b);
                     }
                 } else {
+                    const uint32_t qbar = q_full_bar(n);
                     mbar_arrive_expect_tx(qbar, kQTx);
 #pragma unroll
                     for (int hf = 0; hf < kHalves; ++hf) {
-                        tma_load_4d(smem_q + hf * Plan::kQHalfBytes, &tm_q, qbar, hf * 64, w.h, w.q0, w.b);
-                        if (kHasTQ) tma_load_4d(smem_tq + hf * Plan::kQHalfBytes, &tm_tq, qbar, hf * 64, w.h, w.q0, w.b);
+                        tma_load_4d(dq + hf * Plan::kQHalfBytes, &tm_q, qbar, hf * 64, wi.h, wi.q0, wi.b);
+                        if (kHasTQ) tma_load_4d(dtq + hf * Plan::kQHalfBytes, &tm_tq, qbar, hf * 64, wi.h, wi.q0, wi.b);
                     }
                 }
+            };
+            Item prev_w{};
+            int it = 0;
+            Walk wk = walk_init(first_item);
+            for (int item = first_item; ok && item < n_items; item += item_stride, ++it, walk_step(wk)) {
+                w = item_of(wk);
                 const bool has_next = n_items - item > item_stride;
-                if (has_next) {
-                    // the next item's Q, tQ can only be loaded once this item's score MMAs are done: have them
-                    // waiting in L2 by then
-                    const Item nx = decode(item + item_stride);
+                Walk wk_next = wk;
+                walk_step(wk_next);
+                if (!kDoubleQ) {
+                    // one Q/tQ buffer: it is free once all score MMAs of the item before are complete
+                    if (it > 0) ok = mbar_wait(smem_u32(&bar_q_free), (it - 1) & 1, abort_state);
+                    if (!ok) break;
+                    TRACE(1, it);         // producer: Q, tQ may be replaced
+                    load_q(it, w);
+                    if (has_next) {
+                        // the next item's Q, tQ can only be loaded once this item's score MMAs are done: have them
+                        // waiting in L2 by then
+                        const Item nx = item_of(wk_next);
 #pragma unroll
-                    for (int hf = 0; hf < kHalves; ++hf) {
-                        tma_prefetch_4d(&tm_q, hf * 64, nx.h, nx.q0, nx.b);
-                        if (kHasTQ) tma_prefetch_4d(&tm_tq, hf * 64, nx.h, nx.q0, nx.b);
+                        for (int hf = 0; hf < kHalves; ++hf) {
+                            tma_prefetch_4d(&tm_q, hf * 64, nx.h, nx.q0, nx.b);
+                            if (kHasTQ) tma_prefetch_4d(&tm_tq, hf * 64, nx.h, nx.q0, nx.b);
+                        }
                     }
+                } else if (it == 0) {
+                    load_q(0, w);         // later items: loaded during the item before (below)
                 }
-                for (int t = 0; ok && t < kBufs && t < w.n_kv; ++t) ok = load_k(t);
-#if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 3
-                {   // timing experiment: when do Q, tQ land?
-                    const unsigned long long t0 = globaltimer_ns();
-                    while (!mbar_test_wait(qbar, it & 1) && globaltimer_ns() - t0 < 1000000ull) {}
-                    TRACE(19, it);
+                if (!(stream_items && it > 0)) {
+                    for (int t = 0; ok && t < kBufs && t < w.n_kv; ++t) ok = load_k(t);
                 }
-#endif
                 // staging slots of the item before: after this item's leading K tiles (which the first score MMAs
                 // need at once) and before its V tiles (which are not needed until the first softmax is through)
-                if (kStageSlots > 0 && ok && it > 0) ok = acquire_stage(it - 1, prev_w);
+                if (kRingStage > 0 && ok && it > 0) ok = acquire_stage(it - 1, prev_w);
+                bool next_q_loaded = false;
+                // a leading K tile of the next item (stream_items), in the ring position where the MMA warp consumes it
+                auto load_k_of_next = [&](int t) -> bool {
+                    const Item cur = w;
+                    w = item_of(wk_next);
+                    const bool r = load_k(t);
+                    w = cur;
+                    return r;
+                };
                 for (int j = 0; ok && j < w.n_kv; ++j) {
-                    if (j >= 1 && j + kBufs - 1 < w.n_kv) ok = load_k(j + kBufs - 1);
+                    if (j >= 1) {
+                        const int kn = j + kBufs - 1;        // the K tile consumed after V(j - 1)
+                        if (kn < w.n_kv) ok = load_k(kn);
+                        else if (stream_items && has_next) ok = load_k_of_next(kn - w.n_kv);
+                    }
                     if (ok) ok = load_v(j);
                     // the previous item's outputs: the loads above do not depend on its epilogue, the later ones do
-                    if (ok && stage_pending && (j == 1 || j + 1 == w.n_kv)) ok = store_staged();
+                    if (ok && (j == 1 || j + 1 == w.n_kv)) {
+                        if (stage_pending) ok = store_staged();
+                        if (kDoubleQ && ok && has_next && !next_q_loaded) {
+                            // Two Q/tQ buffers: the other buffer held the item before and then its staged output
+                            // tiles, which the stores above have just read (split-KV stages nothing: there the
+                            // buffer is free once that item's score MMAs are complete).
+                            if (kStageSlots == 0 && it > 0) ok = mbar_wait(smem_u32(&bar_q_free), (it - 1) & 1, abort_state);
+                            if (ok) {
+                                TRACE(1, it + 1);     // producer: Q, tQ buffer of the next item is free
+                                load_q(it + 1, item_of(wk_next));
+                                next_q_loaded = true;
+                            }
+                        }
+                    }
                 }
+                if (ok && stream_items && has_next) ok = load_k_of_next(kBufs - 1);    // consumed after V(n - 1)
                 prev_w = w;
+                if (kDoubleQ && kStageSlots > 0 && ok) {
+                    // this item's output tiles will be staged in its own Q/tQ buffer; stored during the next item
+                    stage_pending = true;
+                    stage_it = it;
+                    stage_w = w;
+                }
                 // the CTA's last item: its staging slots follow its last V tile
-                if (kStageSlots > 0 && ok && !has_next) ok = acquire_stage(it, w);
+                if (kRingStage > 0 && ok && !has_next) ok = acquire_stage(it, w);
             }
             if (ok && stage_pending) ok = store_staged();
             if (kStageSlots > 0) tma_store_wait_all();
@@ -901,8 +991,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             constexpr uint32_t kVLbo = Plan::kKvHalfBytes;   // bytes between 64-wide N atoms of a V slot
             const bool leader = elect_one();
             bool ok = true;
-            const uint32_t q_lo = make_desc_lo(smem_q, 16);
-            const uint32_t tq_lo = make_desc_lo(smem_tq, 16);
+            uint32_t q_lo = make_desc_lo(q_addr(0), 16);     // set per item (two Q/tQ buffers alternate)
+            uint32_t tq_lo = make_desc_lo(tq_addr(0), 16);
 
             // The hardware queue in front of the tensor pipe is short (about eight instructions), and this
             // warp competes for issue slots with the softmax warps, so whatever runs between two
@@ -933,7 +1023,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             constexpr bool kPairRowsOnly = kPair && !kHasTKV;
             constexpr uint32_t kPairOff2 = kHasTKV ? kHalves * Plan::kKvHalfBytes : 0;   // pair: the slot's second region
             auto kd = [&](int k) {
-                return make_desc(k_lo + (((k / 4) * (kPairRowsOnly ? Plan::kKvHalfBytes / 2 : (kPair ? 1 : 2) * Plan::kKvHalfBytes)
+                return make_desc(k_lo + (((k / 4) * (kPairRowsOnly ? Plan::kKvHalfBytes / 2
+                                                     : (kPair ? 1 : Plan::kTilesPerSlot) * Plan::kKvHalfBytes)
                                           + (k % 4) * 32) >> 4));
             };
             // B operand of tQ K^T: the K rows of the same stack; CTA pair: this CTA's 32 rows of K (halves of 4 KB)
@@ -957,16 +1048,16 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
             // score MMAs of global tile g (issued by the elected lane), in two parts so that the look-ahead for
             // the next tile can run between them; `last_of_item`: these are the item's last score MMAs
-            auto issue_scores_a = [&](int g) {
-                const uint32_t tm_s = tmem + kScoreCol0 + sbuf(g) * kScoreBufStride;
+            auto issue_scores_a = [&](int g, int buf) {
+                const uint32_t tm_s = tmem + kScoreCol0 + buf * kScoreBufStride;
                 TRACE(21, g);         // MMA: about to issue score MMAs
                 mma_ss0(tm_s, qd(0), kd(0), kIdescS1);
 #pragma unroll
                 for (int k = 1; k < D / 16; ++k) mma_ss1(tm_s, qd(k), kd(k), kIdescS1);
-                if (kEarlyS) commit(smem_u32(&bar_s_full[sbuf(g)]));     // S is complete; tS follows
+                if (kEarlyS) commit(smem_u32(&bar_s_full[buf]));     // S is complete; tS follows
             };
-            auto issue_scores_b = [&](int g, int slot, bool last_of_item) {
-                const uint32_t tm_ts = tmem + kScoreCol0 + sbuf(g) * kScoreBufStride + kBlockN;
+            auto issue_scores_b = [&](int g, int buf, int slot, bool last_of_item) {
+                const uint32_t tm_ts = tmem + kScoreCol0 + buf * kScoreBufStride + kBlockN;
                 if (kHasTQ) {
                     if (kHasTKV) mma_ss1(tm_ts, tqd(0), k2d(0), kIdescS2);
                     else mma_ss0(tm_ts, tqd(0), k2d(0), kIdescS2);
@@ -974,23 +1065,23 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     for (int k = 1; k < D / 16; ++k) mma_ss1(tm_ts, tqd(k), k2d(k), kIdescS2);
                 }
                 commit(smem_u32(&bar_slot_empty[slot]));
-                commit(smem_u32(kEarlyS ? &bar_ts_full[sbuf(g)] : &bar_s_full[sbuf(g)]));
+                commit(smem_u32(kEarlyS ? &bar_ts_full[buf] : &bar_s_full[buf]));
                 if (last_of_item) commit(smem_u32(&bar_q_free));
                 TRACE(2, g);          // MMA: score MMAs of tile g issued
             };
             // value MMAs of tile j of the item (global tile g) out of ring slot `slot`
             // value MMAs of tile j of the item (global tile g) out of ring slot `slot`, in two parts: those that read
             // P~ can run while the softmax warps are still forming H~
-            auto issue_values_p = [&](int j, int g) {
-                const uint32_t tm_p = tmem + kScoreCol0 + sbuf(g) * kScoreBufStride;
+            auto issue_values_p = [&](int j, int g, int buf) {
+                const uint32_t tm_p = tmem + kScoreCol0 + buf * kScoreBufStride;
                 TRACE(3, g);          // MMA: about to issue value MMAs
 #pragma unroll
                 for (int k = 0; k < kBlockN / 16; ++k) {
                     mma_tsx(tmem_o, tm_p + k * 8, vd(k), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
                 }
             };
-            auto issue_values_h = [&](int j, int g, int slot) {
-                const uint32_t tm_h = tmem + kScoreCol0 + sbuf(g) * kScoreBufStride + kBlockN;
+            auto issue_values_h = [&](int j, int g, int buf, int slot) {
+                const uint32_t tm_h = tmem + kScoreCol0 + buf * kScoreBufStride + kBlockN;
                 if (kHasTQ) {
 #pragma unroll
                     for (int k = 0; k < kBlockN / 16; ++k) {
@@ -1002,31 +1093,40 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 TRACE(4, g);          // MMA: value MMAs of tile g issued
             };
             // what the burst of global tile g needs: V and K(+2) in shared memory, P~/H~ in tensor memory
-            auto test_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, int g) -> bool {
+            auto test_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, const BufPos& bp) -> bool {
                 bool r = mbar_test_wait(smem_u32(&bar_slot_full[pv.slot]), pv.parity);
                 if (has_k) r = r && mbar_test_wait(smem_u32(&bar_slot_full[pk.slot]), pk.parity);
-                r = r && mbar_test_wait(smem_u32(&bar_p_full[sbuf(g)]), sphase(g));
+                r = r && mbar_test_wait(smem_u32(&bar_p_full[bp.buf]), bp.phase);
                 return __all_sync(0xffffffffu, r);
             };
-            auto wait_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, int g) -> bool {
+            auto wait_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, int g, const BufPos& bp) -> bool {
                 if (leader) TRACE(22, g);   // MMA: has to block for tile g
                 bool r = wait_full(pv);
                 if (r && has_k) r = wait_full(pk);
-                if (r) r = mbar_wait_warp(smem_u32(&bar_p_full[sbuf(g)]), sphase(g), abort_state);
+                if (r) r = mbar_wait_warp(smem_u32(&bar_p_full[bp.buf]), bp.phase, abort_state);
                 return r;
             };
 
             // Ring order (as the producer fills it), per item: K0, K1, V0, K2, V1, K3, ...
             RingPos pos{0, 0u};
+            BufPos bp{0, 0u};    // score buffer / phase of the tile whose value MMAs come next
             int g0 = 0;          // global number of the item's first key tile
             int it = 0;
-            for (int item = first_item; ok && item < n_items; item += item_stride, ++it) {
-                const Item w = decode(item);
+            Walk wk = walk_init(first_item);
+            for (int item = first_item; ok && item < n_items; item += item_stride, ++it, walk_step(wk)) {
+                const Item w = item_of(wk);
                 const int n_kv = w.n_kv;
-                ok = mbar_wait_warp(smem_u32(&bar_q_full), it & 1, abort_state);
+                const bool has_next_item = n_items - item > item_stride;
+                // stream_items: this item's leading score MMAs went out with the last bursts of the item before
+                const bool leading_done = stream_items && it > 0;
+                // ... and the next item's go out with the last bursts of this one
+                const bool feeds_next = stream_items && has_next_item;
+                ok = mbar_wait_warp(q_full_bar(it), q_full_phase(it), abort_state);
                 if (leader) TRACE(10, it);    // MMA: Q, tQ of the item seen
+                q_lo = make_desc_lo(q_addr(it), 16);
+                tq_lo = make_desc_lo(tq_addr(it), 16);
                 // the item's leading score MMAs: one tile per score buffer
-                for (int t = 0; ok && t < kBufs && t < n_kv; ++t) {
+                for (int t = leading_done ? kBufs : 0; ok && t < kBufs && t < n_kv; ++t) {
                     ok = wait_full(pos);
                     if (!ok) break;
                     if (t == 0) {
@@ -1034,21 +1134,23 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         tc_fence_after();
                     }
                     prepare_k(pos.slot);
-                    if (leader) { issue_scores_a(g0 + t); issue_scores_b(g0 + t, pos.slot, t + 1 == n_kv); }
+                    // (leading tile t sits t score buffers after the item's first tile: t < kBufs, no phase needed)
+                    const int lbuf = bp.buf + t < kBufs ? bp.buf + t : bp.buf + t - kBufs;
+                    if (leader) { issue_scores_a(g0 + t, lbuf); issue_scores_b(g0 + t, lbuf, pos.slot, t + 1 == n_kv); }
                     __syncwarp();
                     advance(pos);
                 }
                 if (!ok) break;
                 // the ring positions between the item's leading K tiles and V(0) stage the previous item's outputs
-                if (it > 0) { for (int s = 0; s < kStageSlots; ++s) advance(pos); }
+                if (it > 0) { for (int s = 0; s < kRingStage; ++s) advance(pos); }
                 // pos = V(0).  Per tile j: burst = value MMAs of tile j, score MMAs of tile j + kBufs; the barriers of
                 // tile j+1 are tested in the middle of the burst, while the queue is still full.
                 RingPos pos_v = pos, pos_k = pos;
-                bool has_k = n_kv > kBufs;
+                bool has_k = n_kv > kBufs || feeds_next;      // (stream_items implies n_kv >= kBufs)
                 advance(pos);
                 pos_k = pos;
                 if (has_k) advance(pos);
-                ok = wait_tile(pos_v, pos_k, has_k, g0);
+                ok = wait_tile(pos_v, pos_k, has_k, g0, bp);
                 // the first value MMA of an item overwrites O and T: the previous item's epilogue must have read them
                 if (ok && it > 0) ok = mbar_wait_warp(smem_u32(&bar_acc_free), (it - 1) & 1, abort_state);
                 if (!ok) break;
@@ -1059,7 +1161,15 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const RingPos nxt_v = pos;
                     RingPos nxt_k = pos;
                     const bool nxt_exists = j + 1 < n_kv;
-                    const bool nxt_has_k = j + 1 + kBufs < n_kv;
+                    const bool nxt_has_k = j + 1 + kBufs < n_kv || feeds_next;
+                    if (feeds_next && j + kBufs == n_kv) {
+                        // from here on the score MMAs are those of the next item's leading tiles: its Q, tQ (loaded
+                        // during this item into the other buffer)
+                        ok = mbar_wait_warp(q_full_bar(it + 1), q_full_phase(it + 1), abort_state);
+                        if (!ok) break;
+                        q_lo = make_desc_lo(q_addr(it + 1), 16);
+                        tq_lo = make_desc_lo(tq_addr(it + 1), 16);
+                    }
                     if (nxt_exists) {
                         advance(pos);
                         nxt_k = pos;
@@ -1068,12 +1178,14 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (leader) TRACE(29, g0 + j);   // MMA: burst of tile j begins (loop top)
                     tc_fence_after();
                     if (leader) TRACE(30, g0 + j);   // MMA: after the tensor-core fence
-                    if (leader) issue_values_p(j, g0 + j);
+                    BufPos bp_next = bp;
+                    next_buf(bp_next);
+                    if (leader) issue_values_p(j, g0 + j, bp.buf);
                     __syncwarp();
                     if (kSplitHandover) {
                         // H~ follows P~ by a few hundred cycles: normally it is there by now
-                        const uint32_t hbar = smem_u32(&bar_h_full[sbuf(g0 + j)]);
-                        const uint32_t hpar = sphase(g0 + j);
+                        const uint32_t hbar = smem_u32(&bar_h_full[bp.buf]);
+                        const uint32_t hpar = bp.phase;
                         if (!__all_sync(0xffffffffu, mbar_test_wait(hbar, hpar))) {
                             if (leader) TRACE(24, g0 + j);   // MMA: has to block for H~ of tile g
                             ok = mbar_wait_warp(hbar, hpar, abort_state);
@@ -1083,13 +1195,15 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         tc_fence_after();
                     }
                     if (leader) {
-                        issue_values_h(j, g0 + j, pos_v.slot);
-                        if (has_k) issue_scores_a(g0 + j + kBufs);
+                        issue_values_h(j, g0 + j, bp.buf, pos_v.slot);
+                        if (has_k) issue_scores_a(g0 + j + kBufs, bp.buf);    // tile j + kBufs reuses tile j's buffer
                     }
                     __syncwarp();
                     bool nxt_ready = true;
-                    if (nxt_exists) nxt_ready = test_tile(nxt_v, nxt_k, nxt_has_k, g0 + j + 1);
-                    if (leader && has_k) issue_scores_b(g0 + j + kBufs, pos_k.slot, j + kBufs + 1 == n_kv);
+                    if (nxt_exists) nxt_ready = test_tile(nxt_v, nxt_k, nxt_has_k, bp_next);
+                    // (tile j + kBufs of this item, or tile j + kBufs - n_kv of the next one: either way its last tile
+                    // has index n_kv - 1 there, all items being equally long in stream_items)
+                    if (leader && has_k) issue_scores_b(g0 + j + kBufs, bp.buf, pos_k.slot, j + kBufs + 1 == n_kv || j + kBufs + 1 == 2 * n_kv);
                     __syncwarp();
                     if (leader) TRACE(23, g0 + j);   // MMA: burst of tile j issued, warp reconverged
                     // descriptors of the next burst (this warp is held back by the full queue here anyway)
@@ -1097,7 +1211,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         prepare_v(nxt_v.slot);
                         if (nxt_has_k) prepare_k(nxt_k.slot);
                     }
-                    if (nxt_exists && !nxt_ready) ok = wait_tile(nxt_v, nxt_k, nxt_has_k, g0 + j + 1);
+                    if (nxt_exists && !nxt_ready) ok = wait_tile(nxt_v, nxt_k, nxt_has_k, g0 + j + 1, bp_next);
+                    bp = bp_next;
                     pos_v = nxt_v;
                     pos_k = nxt_k;
                     has_k = nxt_has_k;
@@ -1137,6 +1252,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         const bool neg_scale = c1 < 0.0f;
         bool ok = true;
         int g0 = 0;          // global number of the item's first key tile
+        BufPos bp{0, 0u};    // score buffer / phase of tile g0 + j, advanced for every tile (also the other group's)
         int it = 0;
         int ring_slot = 0;   // ring slot of the item's first position (the ring hands out 2 n + kStageSlots per item)
         // exchange area of the two groups, one fp32 per row each
@@ -1152,8 +1268,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             else mbar_arrive(bar);
         };
 
-        for (int item = first_item; ok && item < n_items; item += item_stride, ++it) {
-            const Item w = decode(item);
+        Walk wk = walk_init(first_item);
+        for (int item = first_item; ok && item < n_items; item += item_stride, ++it, walk_step(wk)) {
+            const Item w = item_of(wk);
             const int n_kv = w.n_kv;
             float m_ref = -INFINITY;   // running reference max, log2 domain (m of Algorithm 2, lazily updated)
             float l_run = 0.0f;        // l (two groups: this group's share)
@@ -1165,9 +1282,11 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
             for (int j = 0; j < n_kv; ++j) {
                 const int g = g0 + j;
+                const int bsel = bp.buf;
+                const uint32_t bphase = bp.phase;
+                next_buf(bp);
                 if (kGroups == 2 && (g & 1) != grp) continue;
-                const int bsel = sbuf(g);
-                if (!mbar_wait_warp(smem_u32(&bar_s_full[bsel]), sphase(g), abort_state)) { ok = false; break; }
+                if (!mbar_wait_warp(smem_u32(&bar_s_full[bsel]), bphase, abort_state)) { ok = false; break; }
                 tc_fence_after();
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
                 const bool trace_me = trace_on && lane == 0;
@@ -1324,7 +1443,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (kHasTQ) {
                     if (kEarlyS) {
                         // tS follows S: the MMAs of tQ K^T ran while the exponentials above were computed
-                        if (!mbar_wait_warp(smem_u32(&bar_ts_full[bsel]), sphase(g), abort_state)) { ok = false; break; }
+                        if (!mbar_wait_warp(smem_u32(&bar_ts_full[bsel]), bphase, abort_state)) { ok = false; break; }
                         tc_fence_after();
 #pragma unroll
                         for (int c0 = 0; c0 < kBlockN; c0 += 32) TMEM_LD32(tm_ts + c0, tv, c0);
@@ -1370,9 +1489,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // slots come after the next item's leading K tiles (every item has n_kv tiles here: the kernel that
             // cuts the keys into chunks stages nothing), or right after its last V tile if it is the CTA's last.
             int stage_slot_o = 0;
-            if (kStageSlots > 0) {
+            if (kRingStage > 0) {
                 const bool has_next = n_items - item > item_stride;
-                const int next_start = (ring_slot + 2 * (n_kv % kSlots) + (it > 0 ? kStageSlots : 0)) % kSlots;
+                const int next_start = (ring_slot + 2 * (n_kv % kSlots) + (it > 0 ? kRingStage : 0)) % kSlots;
                 stage_slot_o = has_next ? (next_start + min(kBufs, n_kv)) % kSlots : next_start;
                 ring_slot = next_start;
             }
@@ -1428,9 +1547,14 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // bf16 outputs: staged in the ring slots after the item's last V tile, in the 128-byte-swizzled
             // layout of the output tensor maps (row r, 16-byte chunk c of a 64-column half at r*128 + (c ^ (r&7))*16)
             uint32_t stage_o = 0, stage_t = 0;
-            if (kStageSlots > 0) {
+            if (kRingStage > 0) {
                 stage_o = smem_ring + stage_slot_o * Plan::kSlotBytes + row * 128;
                 stage_t = smem_ring + ((stage_slot_o + 1) % kSlots) * Plan::kSlotBytes + row * 128;
+            } else if (kStageSlots > 0) {
+                // two Q/tQ buffers: the item's own Q and tQ tiles are dead (its last value MMAs are complete, hence
+                // every MMA issued before them) and have the size and layout of its output tiles
+                stage_o = q_addr(it) + row * 128;
+                stage_t = tq_addr(it) + row * 128;
             }
 #pragma unroll 1
             for (int c0 = 0; c0 < D; c0 += 32) {
@@ -1438,7 +1562,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 uint32_t tvv[32];
                 TMEM_LD32(tmem_o + lane_base + c0, ov, 0);
                 if (kHasTQ) TMEM_LD32(tmem_t + lane_base + c0, tvv, 0);
-                if (kStageSlots > 0 && c0 == 0) {
+                if (kRingStage > 0 && c0 == 0) {
                     ok = mbar_wait_warp(smem_u32(&bar_stage_ready), it & 1, abort_state);
                     if (!ok) { tc_wait_ld(); break; }
                 }

@@ -68,6 +68,25 @@ NAMES = {21: "MMA   score MMAs: issue begins", 2: "MMA   score MMAs issued", 3: 
          28: "  softmax P~ stored", 13: "  softmax tile handed back"}
 
 
+ITEM_NAMES = {1: "producer: Q, tQ may be replaced (q_free seen)", 10: "MMA   Q, tQ of the item seen", 11: "MMA   K(0) of the item seen",
+              12: "  softmax epilogue begins", 20: "  softmax epilogue ends", 9: "producer: staging slots handed over",
+              17: "producer: staged tiles complete, stores issued", 18: "producer: staging slots back in the ring"}
+
+
+def report_items(t, first_item=3, count=2, tiles_per_item=8):
+    """Timeline around the hand-over between work items of a persistent CTA (item-indexed events plus the tile
+    events of the items' first and last tiles)."""
+    ev = [(t[e][i], nm + f" (item {i})", i) for e, nm in ITEM_NAMES.items() for i in range(first_item, first_item + count) if t[e][i] > 0]
+    for i in range(first_item, first_item + count):
+        for g in (i * tiles_per_item - 1, i * tiles_per_item, i * tiles_per_item + 1):
+            if 0 <= g < STEPS:
+                ev += [(t[e][g], nm + f" (tile {g})", g) for e, nm in NAMES.items() if t[e][g] > 0]
+    ev.sort()
+    base = ev[0][0] if ev else 0
+    for tm, nm, _ in ev:
+        print(f"{tm - base:8d}  {nm}")
+
+
 def report(t, first=20, count=6):
     ev = [(t[e][g], nm, g) for e, nm in NAMES.items() for g in range(first, first + count) if t[e][g] > 0]
     ev.sort()
@@ -94,8 +113,12 @@ def main():
     ap.add_argument("--groups", type=int, default=0)
     ap.add_argument("--pair", type=int, default=0, help="CTA-pair kernel: 0 library's choice, 1 off, 2 on")
     ap.add_argument("--first", type=int, default=20); ap.add_argument("--count", type=int, default=4)
+    ap.add_argument("--items", action="store_true", help="print the hand-over between work items instead of the tiles")
     a = ap.parse_args()
-    report(run(a.B, a.H, a.Lq, a.Lk, a.D, a.mode, a.groups, pair=a.pair), a.first, a.count)
+    t = run(a.B, a.H, a.Lq, a.Lk, a.D, a.mode, a.groups, pair=a.pair)
+    if a.items:
+        report_items(t, tiles_per_item=(a.Lk + 63) // 64)
+    report(t, a.first, 0 if a.items else a.count)
 
 
 if __name__ == "__main__":
