@@ -339,6 +339,45 @@ __device__ __forceinline__ void mma_ts_pair(uint32_t d_tmem, uint32_t a_tmem, ui
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
+// The same instructions guarded by a per-lane predicate: the issuing warp stays converged (every lane executes the
+// instruction stream, the elected lane alone issues), which keeps its loop out of divergent-branch handling.
+template <bool kAccumulate, bool kPairMma>
+__device__ __forceinline__ void mma_ss_if(uint32_t pred, uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+    if (kPairMma) {
+        asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %4, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                     "@q tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(pred), "r"(kAccumulate ? 1u : 0u) : "memory");
+    } else {
+        asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %4, 0;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+                     "@q tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                     ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(pred), "r"(kAccumulate ? 1u : 0u) : "memory");
+    }
+}
+template <bool kPairMma>
+__device__ __forceinline__ void mma_ts_if(uint32_t pred, uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    if (kPairMma) {
+        asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %5, 0;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                     "@q tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                     ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(pred) : "memory");
+    } else {
+        asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 q, %5, 0;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                     "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                     ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(pred) : "memory");
+    }
+}
+template <bool kPairMma>
+__device__ __forceinline__ void tc_commit_if(uint32_t pred, uint32_t bar) {
+    if (kPairMma) {
+        asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %2, 0;\n\t"
+                     "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n\t}"
+                     ::"r"(bar), "h"(static_cast<uint16_t>(3)), "r"(pred) : "memory");
+    } else {
+        asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+                     "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+                     ::"r"(bar), "r"(pred) : "memory");
+    }
+}
+
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -505,9 +544,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // feeds two tensor pipes, so the issuing warp is no longer what a key tile waits for).  Option: it hands P~
     // over early too, and its softmax warps start on S while the MMAs of tQ K^T are still running (kEarlyS: the
     // scores are published in two steps, S after the stacked chain, tS after the second one).
-    // (Measured with one softmax group: 6 % slower than the plain hand-over, because there the softmax warps'
-    // throughput, not their latency, sets the pace, and the extra wait and fence lengthen their tile.  Kept as a
-    // compile-time option.)
+    // (Measured with one softmax group: 6 % slower than the plain hand-over in the pair, 1 % slower in the
+    // tangent-free one-CTA kernel, because there the softmax warps' throughput, not their latency, sets the pace, and
+    // the extra wait and fence lengthen their tile.  Kept as a compile-time option.)
     constexpr bool kEarlyHandover = false;
     constexpr bool kSplitHandover = kHasTQ && (!kHasTKV || (kPair && kEarlyHandover));
     constexpr bool kEarlyS = kPair && kHasTQ && kGroups == 1 && kEarlyHandover;
@@ -1035,22 +1074,19 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // B operand of H~ V: the V atoms of the same slot; CTA pair: this CTA's one atom of V
             auto v2d = [&](int k) { return kPair ? make_desc(v_lo + ((kPairOff2 + k * 2048) >> 4)) : vd(k); };
             // issue and completion tracking in the form the kernel variant needs
-            auto mma_ss0 = [&](uint32_t d, uint64_t a, uint64_t b, uint32_t idesc) {
-                if (kPair) mma_ss_pair<false>(d, a, b, idesc); else mma_ss<false>(d, a, b, idesc);
-            };
-            auto mma_ss1 = [&](uint32_t d, uint64_t a, uint64_t b, uint32_t idesc) {
-                if (kPair) mma_ss_pair<true>(d, a, b, idesc); else mma_ss<true>(d, a, b, idesc);
-            };
+            const uint32_t lead_pred = leader ? 1u : 0u;     // all lanes run the issue code, this lane's instructions take effect
+            auto mma_ss0 = [&](uint32_t d, uint64_t a, uint64_t b, uint32_t idesc) { mma_ss_if<false, kPair>(lead_pred, d, a, b, idesc); };
+            auto mma_ss1 = [&](uint32_t d, uint64_t a, uint64_t b, uint32_t idesc) { mma_ss_if<true, kPair>(lead_pred, d, a, b, idesc); };
             auto mma_tsx = [&](uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc) {
-                if (kPair) mma_ts_pair(d, a, b, idesc, acc); else mma_ts(d, a, b, idesc, acc);
+                mma_ts_if<kPair>(lead_pred, d, a, b, idesc, acc);
             };
-            auto commit = [&](uint32_t bar) { if (kPair) tc_commit_pair(bar); else tc_commit(bar); };
+            auto commit = [&](uint32_t bar) { tc_commit_if<kPair>(lead_pred, bar); };
 
             // score MMAs of global tile g (issued by the elected lane), in two parts so that the look-ahead for
             // the next tile can run between them; `last_of_item`: these are the item's last score MMAs
             auto issue_scores_a = [&](int g, int buf) {
                 const uint32_t tm_s = tmem + kScoreCol0 + buf * kScoreBufStride;
-                TRACE(21, g);         // MMA: about to issue score MMAs
+                if (leader) TRACE(21, g);         // MMA: about to issue score MMAs
                 mma_ss0(tm_s, qd(0), kd(0), kIdescS1);
 #pragma unroll
                 for (int k = 1; k < D / 16; ++k) mma_ss1(tm_s, qd(k), kd(k), kIdescS1);
@@ -1067,14 +1103,14 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 commit(smem_u32(&bar_slot_empty[slot]));
                 commit(smem_u32(kEarlyS ? &bar_ts_full[buf] : &bar_s_full[buf]));
                 if (last_of_item) commit(smem_u32(&bar_q_free));
-                TRACE(2, g);          // MMA: score MMAs of tile g issued
+                if (leader) TRACE(2, g);          // MMA: score MMAs of tile g issued
             };
             // value MMAs of tile j of the item (global tile g) out of ring slot `slot`
             // value MMAs of tile j of the item (global tile g) out of ring slot `slot`, in two parts: those that read
             // P~ can run while the softmax warps are still forming H~
             auto issue_values_p = [&](int j, int g, int buf) {
                 const uint32_t tm_p = tmem + kScoreCol0 + buf * kScoreBufStride;
-                TRACE(3, g);          // MMA: about to issue value MMAs
+                if (leader) TRACE(3, g);          // MMA: about to issue value MMAs
 #pragma unroll
                 for (int k = 0; k < kBlockN / 16; ++k) {
                     mma_tsx(tmem_o, tm_p + k * 8, vd(k), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
@@ -1090,7 +1126,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
                 commit(smem_u32(&bar_slot_empty[slot]));
                 commit(smem_u32(&bar_pv_done[g & 1]));
-                TRACE(4, g);          // MMA: value MMAs of tile g issued
+                if (leader) TRACE(4, g);          // MMA: value MMAs of tile g issued
             };
             // what the burst of global tile g needs: V and K(+2) in shared memory, P~/H~ in tensor memory
             auto test_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, const BufPos& bp) -> bool {
@@ -1136,8 +1172,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     prepare_k(pos.slot);
                     // (leading tile t sits t score buffers after the item's first tile: t < kBufs, no phase needed)
                     const int lbuf = bp.buf + t < kBufs ? bp.buf + t : bp.buf + t - kBufs;
-                    if (leader) { issue_scores_a(g0 + t, lbuf); issue_scores_b(g0 + t, lbuf, pos.slot, t + 1 == n_kv); }
-                    __syncwarp();
+                    issue_scores_a(g0 + t, lbuf);
+                    issue_scores_b(g0 + t, lbuf, pos.slot, t + 1 == n_kv);
                     advance(pos);
                 }
                 if (!ok) break;
@@ -1180,8 +1216,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (leader) TRACE(30, g0 + j);   // MMA: after the tensor-core fence
                     BufPos bp_next = bp;
                     next_buf(bp_next);
-                    if (leader) issue_values_p(j, g0 + j, bp.buf);
-                    __syncwarp();
+                    issue_values_p(j, g0 + j, bp.buf);
                     if (kSplitHandover) {
                         // H~ follows P~ by a few hundred cycles: normally it is there by now
                         const uint32_t hbar = smem_u32(&bar_h_full[bp.buf]);
@@ -1194,17 +1229,13 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         }
                         tc_fence_after();
                     }
-                    if (leader) {
-                        issue_values_h(j, g0 + j, bp.buf, pos_v.slot);
-                        if (has_k) issue_scores_a(g0 + j + kBufs, bp.buf);    // tile j + kBufs reuses tile j's buffer
-                    }
-                    __syncwarp();
+                    issue_values_h(j, g0 + j, bp.buf, pos_v.slot);
+                    if (has_k) issue_scores_a(g0 + j + kBufs, bp.buf);    // tile j + kBufs reuses tile j's buffer
                     bool nxt_ready = true;
                     if (nxt_exists) nxt_ready = test_tile(nxt_v, nxt_k, nxt_has_k, bp_next);
                     // (tile j + kBufs of this item, or tile j + kBufs - n_kv of the next one: either way its last tile
                     // has index n_kv - 1 there, all items being equally long in stream_items)
-                    if (leader && has_k) issue_scores_b(g0 + j + kBufs, bp.buf, pos_k.slot, j + kBufs + 1 == n_kv || j + kBufs + 1 == 2 * n_kv);
-                    __syncwarp();
+                    if (has_k) issue_scores_b(g0 + j + kBufs, bp.buf, pos_k.slot, j + kBufs + 1 == n_kv || j + kBufs + 1 == 2 * n_kv);
                     if (leader) TRACE(23, g0 + j);   // MMA: burst of tile j issued, warp reconverged
                     // descriptors of the next burst (this warp is held back by the full queue here anyway)
                     if (nxt_exists) {
