@@ -1129,17 +1129,25 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (leader) TRACE(4, g);          // MMA: value MMAs of tile g issued
             };
             // what the burst of global tile g needs: V and K(+2) in shared memory, P~/H~ in tensor memory
-            auto test_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, const BufPos& bp) -> bool {
-                bool r = mbar_test_wait(smem_u32(&bar_slot_full[pv.slot]), pv.parity);
-                if (has_k) r = r && mbar_test_wait(smem_u32(&bar_slot_full[pk.slot]), pk.parity);
-                r = r && mbar_test_wait(smem_u32(&bar_p_full[bp.buf]), bp.phase);
-                return __all_sync(0xffffffffu, r);
+            // The three tests are issued back to back (their latencies overlap) and agreed on with one vote:
+            // bit 0 = the V and K slots are full, bit 1 = P~ (and H~) are in tensor memory.
+            auto test_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, const BufPos& bp) -> uint32_t {
+                const bool tv = mbar_test_wait(smem_u32(&bar_slot_full[pv.slot]), pv.parity);
+                const bool tk = mbar_test_wait(smem_u32(&bar_slot_full[has_k ? pk.slot : pv.slot]), has_k ? pk.parity : pv.parity);
+                const bool tp = mbar_test_wait(smem_u32(&bar_p_full[bp.buf]), bp.phase);
+                if (__all_sync(0xffffffffu, tv & tk & tp)) return 3u;
+                return __all_sync(0xffffffffu, tv & tk) ? 1u : 0u;
             };
-            auto wait_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, int g, const BufPos& bp) -> bool {
+            // blocks for whatever test_tile() did not see (`seen`: its result)
+            auto wait_tile = [&](const RingPos& pv, const RingPos& pk, bool has_k, int g, const BufPos& bp, uint32_t seen) -> bool {
                 if (leader) TRACE(22, g);   // MMA: has to block for tile g
-                bool r = wait_full(pv);
-                if (r && has_k) r = wait_full(pk);
-                if (r) r = mbar_wait_warp(smem_u32(&bar_p_full[bp.buf]), bp.phase, abort_state);
+                bool r = true;
+                if (!(seen & 1u)) {
+                    r = wait_full(pv);
+                    if (r && has_k) r = wait_full(pk);
+                    if (leader) TRACE(19, g);   // MMA: the tile's V and K slots are full
+                }
+                if (r && !(seen & 2u)) r = mbar_wait_warp(smem_u32(&bar_p_full[bp.buf]), bp.phase, abort_state);
                 return r;
             };
 
@@ -1186,18 +1194,13 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 advance(pos);
                 pos_k = pos;
                 if (has_k) advance(pos);
-                ok = wait_tile(pos_v, pos_k, has_k, g0, bp);
+                ok = wait_tile(pos_v, pos_k, has_k, g0, bp, 0u);
                 // the first value MMA of an item overwrites O and T: the previous item's epilogue must have read them
                 if (ok && it > 0) ok = mbar_wait_warp(smem_u32(&bar_acc_free), (it - 1) & 1, abort_state);
                 if (!ok) break;
                 prepare_v(pos_v.slot);
                 if (has_k) prepare_k(pos_k.slot);
                 for (int j = 0; ok && j < n_kv; ++j) {
-                    // ring positions of the next tile
-                    const RingPos nxt_v = pos;
-                    RingPos nxt_k = pos;
-                    const bool nxt_exists = j + 1 < n_kv;
-                    const bool nxt_has_k = j + 1 + kBufs < n_kv || feeds_next;
                     if (feeds_next && j + kBufs == n_kv) {
                         // from here on the score MMAs are those of the next item's leading tiles: its Q, tQ (loaded
                         // during this item into the other buffer)
@@ -1206,16 +1209,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         q_lo = make_desc_lo(q_addr(it + 1), 16);
                         tq_lo = make_desc_lo(tq_addr(it + 1), 16);
                     }
-                    if (nxt_exists) {
-                        advance(pos);
-                        nxt_k = pos;
-                        if (nxt_has_k) advance(pos);
-                    }
                     if (leader) TRACE(29, g0 + j);   // MMA: burst of tile j begins (loop top)
                     tc_fence_after();
                     if (leader) TRACE(30, g0 + j);   // MMA: after the tensor-core fence
-                    BufPos bp_next = bp;
-                    next_buf(bp_next);
                     issue_values_p(j, g0 + j, bp.buf);
                     if (kSplitHandover) {
                         // H~ follows P~ by a few hundred cycles: normally it is there by now
@@ -1231,18 +1227,33 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     }
                     issue_values_h(j, g0 + j, bp.buf, pos_v.slot);
                     if (has_k) issue_scores_a(g0 + j + kBufs, bp.buf);    // tile j + kBufs reuses tile j's buffer
-                    bool nxt_ready = true;
-                    if (nxt_exists) nxt_ready = test_tile(nxt_v, nxt_k, nxt_has_k, bp_next);
+                    // Middle of the burst, the queue in front of the tensor pipe is full: everything the next burst
+                    // needs is worked out here (its ring positions, score buffer, operand descriptors, and a test
+                    // of its barriers), so that after the last score MMA only the commits stand between this
+                    // burst and the next one.
+                    const bool nxt_exists = j + 1 < n_kv;
+                    const bool nxt_has_k = j + 1 + kBufs < n_kv || feeds_next;
+                    const RingPos nxt_v = pos;
+                    RingPos nxt_k = pos;
+                    BufPos bp_next = bp;
+                    next_buf(bp_next);
+                    uint32_t nxt_seen = 3u;
+                    uint32_t v_lo_next = v_lo, k_lo_next = k_lo;
+                    if (nxt_exists) {
+                        advance(pos);
+                        nxt_k = pos;
+                        if (nxt_has_k) advance(pos);
+                        nxt_seen = test_tile(nxt_v, nxt_k, nxt_has_k, bp_next);
+                        v_lo_next = make_desc_lo(smem_ring + nxt_v.slot * Plan::kSlotBytes, kVLbo);
+                        if (nxt_has_k) k_lo_next = make_desc_lo(smem_ring + nxt_k.slot * Plan::kSlotBytes, 16);
+                    }
                     // (tile j + kBufs of this item, or tile j + kBufs - n_kv of the next one: either way its last tile
                     // has index n_kv - 1 there, all items being equally long in stream_items)
                     if (has_k) issue_scores_b(g0 + j + kBufs, bp.buf, pos_k.slot, j + kBufs + 1 == n_kv || j + kBufs + 1 == 2 * n_kv);
-                    if (leader) TRACE(23, g0 + j);   // MMA: burst of tile j issued, warp reconverged
-                    // descriptors of the next burst (this warp is held back by the full queue here anyway)
-                    if (nxt_exists) {
-                        prepare_v(nxt_v.slot);
-                        if (nxt_has_k) prepare_k(nxt_k.slot);
-                    }
-                    if (nxt_exists && !nxt_ready) ok = wait_tile(nxt_v, nxt_k, nxt_has_k, g0 + j + 1, bp_next);
+                    if (leader) TRACE(23, g0 + j);   // MMA: burst of tile j issued
+                    if (nxt_seen != 3u) ok = wait_tile(nxt_v, nxt_k, nxt_has_k, g0 + j + 1, bp_next, nxt_seen);
+                    v_lo = v_lo_next;
+                    k_lo = k_lo_next;
                     bp = bp_next;
                     pos_v = nxt_v;
                     pos_k = nxt_k;
