@@ -34,6 +34,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     tmp = LIB + f".tmp{os.getpid()}"
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-o", tmp, SRC, "-lcudart"]
+    cmd[1:1] = os.environ.get("ATTN_JVP_NVCC_EXTRA", "").split()     # e.g. -DATTN_JVP_DEBUG
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

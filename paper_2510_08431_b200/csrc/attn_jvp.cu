@@ -337,7 +337,9 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     ka.Lk = Lk;
     ka.n_kv_tiles = (Lk + attn_jvp::kBlockN - 1) / attn_jvp::kBlockN;
     ka.scale = scale;
-    ka.scale_log2 = scale * 1.4426950408889634f;
+    // The kernel masks the keys past Lk by setting their scaled score to -inf, which needs a nonzero factor: a zero
+    // scale (every score 0) is computed with 2^-100 in the exponent, which changes no result bit (tS keeps the 0).
+    ka.scale_log2 = (scale == 0.0f) ? 0x1p-100f : scale * 1.4426950408889634f;
     ka.mu = mu;
     ka.B = B;
     ka.splits = eff_splits;

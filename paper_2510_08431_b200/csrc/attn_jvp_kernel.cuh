@@ -71,6 +71,18 @@ __device__ long long g_trace[kTraceEvents][kTraceSteps];
 #else
 #define TRACE(evt, idx) do { } while (0)
 #endif
+// Totals per role (both trace levels): cycles spent blocked, summed in a register and written once at the end.
+#ifdef ATTN_JVP_TRACE
+#define ACC_DECL(v) long long v = 0, v##_n = 0
+#define ACC_BEGIN(v) const long long v##_t0 = clock64()
+#define ACC_END(v) do { v += clock64() - v##_t0; ++v##_n; } while (0)
+#define ACC_WRITE(slot, v) do { if (trace_on && lane == 0) { g_trace[kTraceEvents - 2][2 * (slot)] = v; g_trace[kTraceEvents - 2][2 * (slot) + 1] = v##_n; } } while (0)
+#else
+#define ACC_DECL(v) do { } while (0)
+#define ACC_BEGIN(v) do { } while (0)
+#define ACC_END(v) do { } while (0)
+#define ACC_WRITE(slot, v) do { } while (0)
+#endif
 
 // Set by any kernel whose bounded wait expired; later CTAs see it and leave at once.
 __device__ int g_abort_flag = 0;
@@ -536,20 +548,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // fp32 partial results straight from registers and stages nothing.
     constexpr int kStageSlots = kSplit ? 0 : (kHasTQ ? 2 : 1);       // output tiles staged per item ...
     constexpr int kRingStage = kDoubleQ ? 0 : kStageSlots;           // ... of which in ring slots (else in the item's Q/tQ buffer)
-    // With tK = tV = 0 the tensor pipe has spare time and a key tile takes as long as the chain softmax -> value
-    // MMAs -> score MMAs: there P~ is handed to the MMA warp as soon as it is stored, and the MMAs that read it run
-    // beside the H~ arithmetic (H~ follows through a barrier of its own).  In the full mode the MMA warp never
-    // waits for the softmax warps, and the second hand-over would only add work (measured: 1 % slower).
-    // The CTA pair runs at the pace of the chain score MMAs -> softmax -> value MMAs as well (one instruction stream
-    // feeds two tensor pipes, so the issuing warp is no longer what a key tile waits for).  Option: it hands P~
-    // over early too, and its softmax warps start on S while the MMAs of tQ K^T are still running (kEarlyS: the
-    // scores are published in two steps, S after the stacked chain, tS after the second one).
-    // (Measured with one softmax group: 6 % slower than the plain hand-over in the pair, 1 % slower in the
-    // tangent-free one-CTA kernel, because there the softmax warps' throughput, not their latency, sets the pace, and
-    // the extra wait and fence lengthen their tile.  Kept as a compile-time option.)
-    constexpr bool kEarlyHandover = false;
-    constexpr bool kSplitHandover = kHasTQ && (!kHasTKV || (kPair && kEarlyHandover));
-    constexpr bool kEarlyS = kPair && kHasTQ && kGroups == 1 && kEarlyHandover;
+    // P~ and H~ of a tile are handed to the MMA warp together (one barrier): the softmax warps form both in one
+    // pass over the columns, so an earlier hand-over of P~ alone would gain nothing.
     constexpr int kBufs = score_buffers(D, MODE);            // score buffers = how many tiles the score MMAs run ahead
     constexpr int kScoreCol0 = (kBufs == 3) ? 128 : 256;     // first column of score buffer 0
     static_assert(kScoreCol0 + kBufs * kScoreBufStride <= kTmemCols, "score buffers must fit into tensor memory");
@@ -562,9 +562,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     __shared__ __align__(8) uint64_t bar_slot_full[kSlots];
     __shared__ __align__(8) uint64_t bar_slot_empty[kSlots];
     __shared__ __align__(8) uint64_t bar_s_full[kBufs];
-    __shared__ __align__(8) uint64_t bar_ts_full[kBufs];    // kEarlyS: tS of the tile is complete (bar_s_full then means S alone)
-    __shared__ __align__(8) uint64_t bar_p_full[kBufs];     // P~ of the tile is in tensor memory
-    __shared__ __align__(8) uint64_t bar_h_full[kBufs];     // H~ of the tile is in tensor memory (some 500 cycles later)
+    __shared__ __align__(8) uint64_t bar_p_full[kBufs];     // P~ and H~ of the tile are in tensor memory
     __shared__ __align__(8) uint64_t bar_pv_done[2];        // the value MMAs of tile g (and all before) are complete: [g & 1]
     __shared__ __align__(8) uint64_t bar_acc_free;   // the epilogue has read O and T: the next item may overwrite them
     __shared__ __align__(8) uint64_t bar_drain;
@@ -678,10 +676,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         for (int i = 0; i < kBufs; ++i) {
             mbar_init(smem_u32(&bar_s_full[i]), 1);
-            mbar_init(smem_u32(&bar_ts_full[i]), 1);
             // one arrival per softmax warp of the tile's group (CTA pair: of both CTAs, on the first CTA's barrier)
             mbar_init(smem_u32(&bar_p_full[i]), (kPair ? 2 : 1) * kSoftmaxThreads / 32);
-            mbar_init(smem_u32(&bar_h_full[i]), (kPair ? 2 : 1) * kSoftmaxThreads / 32);
         }
         mbar_init(smem_u32(&bar_pv_done[0]), 1);
         mbar_init(smem_u32(&bar_pv_done[1]), 1);
@@ -698,7 +694,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #ifdef ATTN_JVP_DEBUG
         if (blockIdx.x == 0) {
             const void* named[] = {&bar_q_full[0], &bar_q_free, &bar_slot_full[0], &bar_slot_empty[0], &bar_s_full[0],
-                                   &bar_p_full[0], &bar_h_full[0], &bar_pv_done[0], &bar_acc_free, &bar_drain,
+                                   &bar_p_full[0], &bar_p_full[0], &bar_pv_done[0], &bar_acc_free, &bar_drain,
                                    &bar_stage_ready, &bar_stage_full, &bar_m[0], &bar_fin[0]};
             for (int i = 0; i < 14; ++i) g_barrier_layout[i] = smem_u32(named[i]);
         }
@@ -746,7 +742,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     const uint32_t tmem_t = tmem + D;
 
     // Phases.  Key tiles are numbered g = 0, 1, 2, ... over ALL items of this CTA; tile g uses score buffer
-    // g % kBufs, phase (g / kBufs) & 1 of bar_s_full / bar_p_full / bar_h_full, and phase (g >> 1) & 1 of
+    // g % kBufs, phase (g / kBufs) & 1 of bar_s_full / bar_p_full, and phase (g >> 1) & 1 of
     // bar_pv_done[g & 1] (two barriers, so that a wait for tile g - 1 cannot be mistaken for one two tiles on).  Item number `it` (0, 1, ...)
     // uses phase it & 1 of bar_q_full / bar_q_free / bar_acc_free / bar_stage_ready / bar_stage_full.  The
     // shared-memory ring runs on without a break; per item it hands out 2 n slots to K/V tiles and then
@@ -1090,7 +1086,6 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 mma_ss0(tm_s, qd(0), kd(0), kIdescS1);
 #pragma unroll
                 for (int k = 1; k < D / 16; ++k) mma_ss1(tm_s, qd(k), kd(k), kIdescS1);
-                if (kEarlyS) commit(smem_u32(&bar_s_full[buf]));     // S is complete; tS follows
             };
             auto issue_scores_b = [&](int g, int buf, int slot, bool last_of_item) {
                 const uint32_t tm_ts = tmem + kScoreCol0 + buf * kScoreBufStride + kBlockN;
@@ -1101,13 +1096,12 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     for (int k = 1; k < D / 16; ++k) mma_ss1(tm_ts, tqd(k), k2d(k), kIdescS2);
                 }
                 commit(smem_u32(&bar_slot_empty[slot]));
-                commit(smem_u32(kEarlyS ? &bar_ts_full[buf] : &bar_s_full[buf]));
+                commit(smem_u32(&bar_s_full[buf]));
                 if (last_of_item) commit(smem_u32(&bar_q_free));
                 if (leader) TRACE(2, g);          // MMA: score MMAs of tile g issued
             };
-            // value MMAs of tile j of the item (global tile g) out of ring slot `slot`
-            // value MMAs of tile j of the item (global tile g) out of ring slot `slot`, in two parts: those that read
-            // P~ can run while the softmax warps are still forming H~
+            // value MMAs of tile j of the item (global tile g) out of ring slot `slot`: those that read P~, then
+            // those that read H~
             auto issue_values_p = [&](int j, int g, int buf) {
                 const uint32_t tm_p = tmem + kScoreCol0 + buf * kScoreBufStride;
                 if (leader) TRACE(3, g);          // MMA: about to issue value MMAs
@@ -1152,6 +1146,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             };
 
             // Ring order (as the producer fills it), per item: K0, K1, V0, K2, V1, K3, ...
+            ACC_DECL(acc_mma_tile);     // blocked for a tile's barriers inside an item
+            ACC_DECL(acc_mma_item);     // blocked at an item's start (first V and K tiles, first P~, accumulators free)
             RingPos pos{0, 0u};
             BufPos bp{0, 0u};    // score buffer / phase of the tile whose value MMAs come next
             int g0 = 0;          // global number of the item's first key tile
@@ -1194,9 +1190,11 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 advance(pos);
                 pos_k = pos;
                 if (has_k) advance(pos);
+                ACC_BEGIN(acc_mma_item);
                 ok = wait_tile(pos_v, pos_k, has_k, g0, bp, 0u);
                 // the first value MMA of an item overwrites O and T: the previous item's epilogue must have read them
                 if (ok && it > 0) ok = mbar_wait_warp(smem_u32(&bar_acc_free), (it - 1) & 1, abort_state);
+                ACC_END(acc_mma_item);
                 if (!ok) break;
                 prepare_v(pos_v.slot);
                 if (has_k) prepare_k(pos_k.slot);
@@ -1213,18 +1211,6 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     tc_fence_after();
                     if (leader) TRACE(30, g0 + j);   // MMA: after the tensor-core fence
                     issue_values_p(j, g0 + j, bp.buf);
-                    if (kSplitHandover) {
-                        // H~ follows P~ by a few hundred cycles: normally it is there by now
-                        const uint32_t hbar = smem_u32(&bar_h_full[bp.buf]);
-                        const uint32_t hpar = bp.phase;
-                        if (!__all_sync(0xffffffffu, mbar_test_wait(hbar, hpar))) {
-                            if (leader) TRACE(24, g0 + j);   // MMA: has to block for H~ of tile g
-                            ok = mbar_wait_warp(hbar, hpar, abort_state);
-                            if (leader) TRACE(25, g0 + j);   // MMA: H~ of tile g seen
-                            if (!ok) break;
-                        }
-                        tc_fence_after();
-                    }
                     issue_values_h(j, g0 + j, bp.buf, pos_v.slot);
                     if (has_k) issue_scores_a(g0 + j + kBufs, bp.buf);    // tile j + kBufs reuses tile j's buffer
                     // Middle of the burst, the queue in front of the tensor pipe is full: everything the next burst
@@ -1251,7 +1237,11 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     // has index n_kv - 1 there, all items being equally long in stream_items)
                     if (has_k) issue_scores_b(g0 + j + kBufs, bp.buf, pos_k.slot, j + kBufs + 1 == n_kv || j + kBufs + 1 == 2 * n_kv);
                     if (leader) TRACE(23, g0 + j);   // MMA: burst of tile j issued
-                    if (nxt_seen != 3u) ok = wait_tile(nxt_v, nxt_k, nxt_has_k, g0 + j + 1, bp_next, nxt_seen);
+                    if (nxt_seen != 3u) {
+                        ACC_BEGIN(acc_mma_tile);
+                        ok = wait_tile(nxt_v, nxt_k, nxt_has_k, g0 + j + 1, bp_next, nxt_seen);
+                        ACC_END(acc_mma_tile);
+                    }
                     v_lo = v_lo_next;
                     k_lo = k_lo_next;
                     bp = bp_next;
@@ -1261,6 +1251,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 }
                 g0 += n_kv;
             }
+            ACC_WRITE(0, acc_mma_tile);
+            ACC_WRITE(1, acc_mma_item);
             if (!ok && leader) {
                 // Abandoning the work: wait (bounded) until the tensor core has drained what was issued.
                 commit(smem_u32(&bar_drain));
@@ -1310,6 +1302,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             else mbar_arrive(bar);
         };
 
+        ACC_DECL(acc_sm_scores);   // blocked for a tile's scores
+        ACC_DECL(acc_sm_values);   // blocked for the item's last value MMAs (epilogue)
+        ACC_DECL(acc_sm_epi);      // epilogue after that wait
         Walk wk = walk_init(first_item);
         for (int item = first_item; ok && item < n_items; item += item_stride, ++it, walk_step(wk)) {
             const Item w = item_of(wk);
@@ -1328,7 +1323,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const uint32_t bphase = bp.phase;
                 next_buf(bp);
                 if (kGroups == 2 && (g & 1) != grp) continue;
+                ACC_BEGIN(acc_sm_scores);
                 if (!mbar_wait_warp(smem_u32(&bar_s_full[bsel]), bphase, abort_state)) { ok = false; break; }
+                ACC_END(acc_sm_scores);
                 tc_fence_after();
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
                 const bool trace_me = trace_on && lane == 0;
@@ -1339,12 +1336,15 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
                 uint32_t sv[kBlockN];
                 uint32_t tv[kBlockN];
+                // S first; tS is fetched while the row maximum is formed
 #pragma unroll
-                for (int c0 = 0; c0 < kBlockN; c0 += 32) {
-                    TMEM_LD32(tm_s + c0, sv, c0);
-                    if (kHasTQ && !kEarlyS) TMEM_LD32(tm_ts + c0, tv, c0);
+                for (int c0 = 0; c0 < kBlockN; c0 += 32) TMEM_LD32(tm_s + c0, sv, c0);
+                if (kGroups == 1 || !kHasTQ) tc_wait_ld();
+                if (kHasTQ) {
+#pragma unroll
+                    for (int c0 = 0; c0 < kBlockN; c0 += 32) TMEM_LD32(tm_ts + c0, tv, c0);
                 }
-                tc_wait_ld();
+                if (kGroups == 2 && kHasTQ) tc_wait_ld();      // (two groups hide the latency by themselves: one wait)
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
                 if (trace_me && quarter == 0 && g < kTraceSteps) g_trace[26][g] = clock64();    // softmax: scores in registers
 #endif
@@ -1404,19 +1404,24 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const int n_valid = valid < kBlockN ? valid : kBlockN;
                     return sc * ((sm4[0] + sm4[1]) + (sm4[2] + sm4[3])) / static_cast<float>(n_valid);
                 };
-                if (kHasTQ && !kEarlyS && j == 0) ts_shift = centre_of_first_tile();
+                if (kHasTQ && kGroups == 1) tc_wait_ld();      // tS is in registers
+                if (kHasTQ && j == 0) ts_shift = centre_of_first_tile();
 
                 // m_new = max(m, rowmax), applied lazily: the result does not depend on which
                 // reference is used as long as exp() stays in range.
-                float alpha = 1.0f;
                 const bool need = mx > m_ref + kRescaleThreshold;
-                if (need) {
-                    alpha = ex2f(m_ref - mx);    // e^{m - m_new}; 0 on the first tile (m = -inf)
-                    m_ref = mx;
-                }
-                if (j > 0 && __any_sync(0xffffffffu, need)) {
+                const float alpha = need ? ex2f(m_ref - mx) : 1.0f;    // e^{m - m_new}; 0 on the first tile (m = -inf)
+                m_ref = need ? mx : m_ref;
+                // (whether any row of the warp rescales: asked here, acted on after the pass over the columns, so that
+                // the vote's latency and the branch stay off the path to the first exponential)
+                const bool any_need = j > 0 && __any_sync(0xffffffffu, need);
+                // Rescale of the accumulators where the reference moved (rare: once or twice per row).  One softmax
+                // group: after the pass over the columns (the branch and the vote's latency stay off the path to the
+                // first exponential); two groups with tangents: before it (their register budget is tighter, and the packed P~, H~
+                // would have to live across the branch).
+                auto rescale_accumulators = [&]() -> bool {
                     // the accumulators must be complete up to tile j-1 before they are rescaled
-                    if (!mbar_wait_warp(smem_u32(&bar_pv_done[(g - 1) & 1]), ((g - 1) >> 1) & 1, abort_state)) { ok = false; break; }
+                    if (!mbar_wait_warp(smem_u32(&bar_pv_done[(g - 1) & 1]), ((g - 1) >> 1) & 1, abort_state)) return false;
                     tc_fence_after();
                     constexpr int kAccCols = kHasTQ ? 2 * D : D;
 #pragma unroll 1
@@ -1428,7 +1433,10 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         for (int c = 0; c < 32; ++c) acc[c] = __float_as_uint(__uint_as_float(acc[c]) * alpha);
                         TMEM_ST32(tmem_o + lane_base + c0, acc, 0);
                     }
-                }
+                    return true;
+                };
+                constexpr bool kLateRescale = (kGroups == 1) || !kHasTQ;
+                if (!kLateRescale && any_need && !rescale_accumulators()) { ok = false; break; }
                 l_run *= alpha;
                 r_run *= alpha;
                 if (kGroups == 2) {
@@ -1439,88 +1447,69 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (lane == 0) mbar_arrive(mbar);
                 }
 
-                // P~ = exp(S - m_new), l += rowsum(P~)   (two columns per FMA-pipe instruction)
+                // P~ = exp(S - m_new), l += rowsum(P~), H~ = P~ . tS, r += rowsum(H~), and both rounded to bf16, in ONE
+                // pass over the columns (two columns per FMA-pipe instruction).  The exponentials set the pace of the
+                // pass (the special-function unit takes 8 cycles per warp instruction, 64 of them per tile), and
+                // everything else fits into the issue slots they leave free; as separate passes the H~ arithmetic
+                // and the conversions came on top.
                 const uint64_t c1c1 = pack_f32x2(c1, c1);
                 const uint64_t negm = pack_f32x2(-m_ref, -m_ref);
-                uint64_t ls2[2] = {0ull, 0ull};     // (+0.0f, +0.0f)
-#pragma unroll
-                for (int c = 0; c < kBlockN; c += 2) {
-                    float x0, x1;
-                    unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), c1c1, negm), x0, x1);
-                    const float p0 = ex2f(x0), p1 = ex2f(x1);
-                    sv[c] = __float_as_uint(p0);
-                    sv[c + 1] = __float_as_uint(p1);
-                    ls2[(c >> 1) & 1] = add_f32x2(ls2[(c >> 1) & 1], pack_f32x2(p0, p1));
-                }
-                float ls4[4];
-                unpack_f32x2(ls2[0], ls4[0], ls4[1]);
-                unpack_f32x2(ls2[1], ls4[2], ls4[3]);
-                if (valid < kBlockN) {
-                    // exact zeros for masked keys whatever the scale (0 * inf above would give NaN)
-                    ls4[0] = ls4[1] = ls4[2] = ls4[3] = 0.0f;
-#pragma unroll
-                    for (int c = 0; c < kBlockN; ++c) {
-                        if (c >= valid) sv[c] = 0u;
-                        ls4[c & 3] += __uint_as_float(sv[c]);
-                    }
-                }
-                const float lsum = (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
-                l_run += lsum;
-                {
-                    uint32_t pk[kBlockN / 2];
-#pragma unroll
-                    for (int c = 0; c < kBlockN / 2; ++c) pk[c] = pack_bf16(__uint_as_float(sv[2 * c]), __uint_as_float(sv[2 * c + 1]));
-                    TMEM_ST32(tm_s, pk, 0);
-                }
+                const uint64_t scsc = pack_f32x2(sc, sc);
+                const uint64_t negshift = pack_f32x2(-ts_shift, -ts_shift);
+                uint32_t pk_p[kBlockN / 2];
+                uint32_t pk_h[kBlockN / 2];
+                float lsum, rsum = 0.0f;
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
-                if (trace_me && quarter == 0 && g < kTraceSteps) g_trace[28][g] = clock64();    // softmax: P~ store issued
+                if (trace_me && quarter == 0 && g < kTraceSteps) g_trace[24][g] = clock64();    // softmax: the pass over the columns begins
 #endif
-                if (kSplitHandover) {
-                    // P~ is handed over at once: the MMAs that read it run beside the H~ arithmetic below
-                    tc_wait_st();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) arrive_at_issuer(smem_u32(&bar_p_full[bsel]));
-                }
-                if (kHasTQ) {
-                    if (kEarlyS) {
-                        // tS follows S: the MMAs of tQ K^T ran while the exponentials above were computed
-                        if (!mbar_wait_warp(smem_u32(&bar_ts_full[bsel]), bphase, abort_state)) { ok = false; break; }
-                        tc_fence_after();
-#pragma unroll
-                        for (int c0 = 0; c0 < kBlockN; c0 += 32) TMEM_LD32(tm_ts + c0, tv, c0);
-                        tc_wait_ld();
-                        if (j == 0) ts_shift = centre_of_first_tile();
-                    }
-                    // H~ = P~ . tS, r += rowsum(H~)
-                    const uint64_t scsc = pack_f32x2(sc, sc);
-                    const uint64_t negshift = pack_f32x2(-ts_shift, -ts_shift);
+                // (Keys past Lk of the item's ragged last tile: their S was set to -inf after scaling above, so P~ is
+                // exactly 0 whatever the scale, the host having replaced a zero scale by 2^-100; their tS is exactly
+                // 0, hence H~ = 0 * (-shift) = 0.)
+                {
+                    uint64_t ls2[2] = {0ull, 0ull};     // (+0.0f, +0.0f)
                     uint64_t rs2[2] = {0ull, 0ull};
 #pragma unroll
                     for (int c = 0; c < kBlockN; c += 2) {
-                        const uint64_t ts2 = fma_f32x2(pack_f32x2(__uint_as_float(tv[c]), __uint_as_float(tv[c + 1])), scsc, negshift);
-                        const uint64_t h2 = mul_f32x2(pack_f32x2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), ts2);
-                        float h0, h1;
-                        unpack_f32x2(h2, h0, h1);
-                        tv[c] = __float_as_uint(h0);
-                        tv[c + 1] = __float_as_uint(h1);
-                        rs2[(c >> 1) & 1] = add_f32x2(rs2[(c >> 1) & 1], h2);
+                        float x0, x1;
+                        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), c1c1, negm), x0, x1);
+                        const float p0 = ex2f(x0), p1 = ex2f(x1);
+                        const uint64_t p2 = pack_f32x2(p0, p1);
+                        ls2[(c >> 1) & 1] = add_f32x2(ls2[(c >> 1) & 1], p2);
+                        pk_p[c >> 1] = pack_bf16(p0, p1);
+                        if (kHasTQ) {
+                            const uint64_t ts2 = fma_f32x2(pack_f32x2(__uint_as_float(tv[c]), __uint_as_float(tv[c + 1])), scsc, negshift);
+                            const uint64_t h2 = mul_f32x2(p2, ts2);
+                            float h0, h1;
+                            unpack_f32x2(h2, h0, h1);
+                            rs2[(c >> 1) & 1] = add_f32x2(rs2[(c >> 1) & 1], h2);
+                            pk_h[c >> 1] = pack_bf16(h0, h1);
+                        }
                     }
-                    {
-                        float a0, a1, a2, a3;
+                    float a0, a1, a2, a3;
+                    unpack_f32x2(ls2[0], a0, a1);
+                    unpack_f32x2(ls2[1], a2, a3);
+                    lsum = (a0 + a1) + (a2 + a3);
+                    if (kHasTQ) {
                         unpack_f32x2(rs2[0], a0, a1);
                         unpack_f32x2(rs2[1], a2, a3);
-                        r_run += (a0 + a1) + (a2 + a3);
+                        rsum = (a0 + a1) + (a2 + a3);
                     }
-                    uint32_t pk[kBlockN / 2];
-#pragma unroll
-                    for (int c = 0; c < kBlockN / 2; ++c) pk[c] = pack_bf16(__uint_as_float(tv[2 * c]), __uint_as_float(tv[2 * c + 1]));
-                    TMEM_ST32(tm_ts, pk, 0);
                 }
+                l_run += lsum;
+                r_run += rsum;
+                if (kLateRescale && any_need && !rescale_accumulators()) { ok = false; break; }
+#if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
+                if (trace_me && quarter == 0 && g < kTraceSteps) g_trace[25][g] = clock64();    // softmax: ... and ends
+#endif
+                TMEM_ST32(tm_s, pk_p, 0);
+                if (kHasTQ) TMEM_ST32(tm_ts, pk_h, 0);
+#if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
+                if (trace_me && quarter == 0 && g < kTraceSteps) g_trace[28][g] = clock64();    // softmax: P~, H~ stores issued
+#endif
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) arrive_at_issuer(smem_u32(kSplitHandover ? &bar_h_full[bsel] : &bar_p_full[bsel]));
+                if (lane == 0) arrive_at_issuer(smem_u32(&bar_p_full[bsel]));
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
                 if (trace_me && g < kTraceSteps) g_trace[13 + ((warp - kFirstSoftmaxWarp) & 3)][g] = clock64();    // softmax warp: arrived
 #endif
@@ -1557,6 +1546,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // them: the value MMAs up to tile g_last - kBufs, and for an item's leading tiles those of all earlier
             // items.  That covers g_last - 3, so tile g_last - 1 can be waited for first, and g_last after it.
             const int g_last = g0 + n_kv - 1;
+            ACC_BEGIN(acc_sm_values);
             if (n_kv >= 2) ok = mbar_wait_warp(smem_u32(&bar_pv_done[(g_last - 1) & 1]), ((g_last - 1) >> 1) & 1, abort_state);
             if (ok) ok = mbar_wait_warp(smem_u32(&bar_pv_done[g_last & 1]), (g_last >> 1) & 1, abort_state);
             if (ok && kGroups == 2) {
@@ -1570,6 +1560,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (lane == 0) mbar_arrive(smem_u32(&bar_fin_read[quarter]));
                 }
             }
+            ACC_END(acc_sm_values);
+            ACC_BEGIN(acc_sm_epi);
             if (!ok) break;
             tc_fence_after();
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
@@ -1678,7 +1670,13 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     if (args.mu != nullptr) args.mu[idx] = mu_val;
                 }
             }
+            ACC_END(acc_sm_epi);
             g0 += n_kv;
+        }
+        if (warp == kFirstSoftmaxWarp + ((kMmaWarp - kFirstSoftmaxWarp) & 3)) {   // the softmax warp on the MMA warp's scheduler
+            ACC_WRITE(2, acc_sm_scores);
+            ACC_WRITE(3, acc_sm_values);
+            ACC_WRITE(4, acc_sm_epi);
         }
     }
 

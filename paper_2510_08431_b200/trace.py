@@ -63,9 +63,9 @@ def run(B, H, Lq, Lk, D, mode="jvp", groups=0, first=20, count=6, seed=4, pair=0
 
 NAMES = {21: "MMA   score MMAs: issue begins", 2: "MMA   score MMAs issued", 3: "MMA   value MMAs: issue begins",
          4: "MMA   value MMAs issued", 29: "MMA   burst begins (loop top)", 30: "MMA   after tensor-core fence",
-         23: "MMA   burst issued, warp reconverged", 19: "MMA   (blocked) V and K slots seen full", 22: "MMA   blocks for the tile's barriers", 24: "MMA   blocks for H~",
+         23: "MMA   burst issued, warp reconverged", 19: "MMA   (blocked) V and K slots seen full", 22: "MMA   blocks for the tile's barriers", 24: "  softmax pass over the columns begins", 25: "  softmax pass over the columns ends",
          5: "  softmax scores seen (s_full)", 26: "  softmax scores in registers", 27: "  softmax reference max agreed",
-         28: "  softmax P~ stored", 13: "  softmax tile handed back"}
+         28: "  softmax P~, H~ stores issued", 13: "  softmax tile handed back"}
 
 
 ITEM_NAMES = {1: "producer: Q, tQ may be replaced (q_free seen)", 10: "MMA   Q, tQ of the item seen", 11: "MMA   K(0) of the item seen",
