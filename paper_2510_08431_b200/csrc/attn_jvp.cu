@@ -60,32 +60,32 @@ int softmax_groups_for_pair(int mode) {
 }
 
 // Whether a call runs on the CTA-pair kernel (clusters of two CTAs sharing the K/V operand tiles and one MMA
-// instruction stream).  It exists for the full JVP at D = 128.
+// instruction stream).  It exists at D = 128, without key chunks.
 bool use_cta_pair(int mode, int D, bool split, int tiles_per_item) {
     if (D != 128 || split) return false;
     const int forced = g_tune_cta_pair.load(std::memory_order_relaxed);
     if (forced == 1) return false;
     if (forced == 2) return true;
-    // Measured on B200.  Full JVP: 4-20 % faster than one CTA per query tile from about eight key tiles per item on
-    // (12 % on the 32760-token self-attention workloads), 4 % slower with two key tiles per item.  Forward only:
-    // 7-9 % faster (with two softmax groups) on the image- and video-length workloads, slower on short items.
-    // Tangent-free K/V: 3-6 % slower everywhere, so it stays on one CTA per query tile.
+    // Measured on B200.  Full JVP: 2-20 % faster than one CTA per query tile from about eight key tiles per item on
+    // (12 % on the 32760-token self-attention workloads), slower with fewer.  Tangent-free K/V: 4-20 % faster from
+    // two key tiles per item on (6 % on the 512-key cross-attention workload, 9 % at 32760 keys).  Forward only:
+    // 4-9 % slower than one CTA per query tile with two softmax groups at every length tried (64 to 32760 keys).
     if (mode == attn_jvp::kModeJvp) return tiles_per_item >= 6;
-    if (mode == attn_jvp::kModeFwdOnly) return tiles_per_item >= 32;
+    if (mode == attn_jvp::kModeKvTangentFree) return tiles_per_item >= 2;
     return false;
 }
 
 // Softmax warpgroups per CTA for a kernel variant: two groups take alternate key tiles, which pays where the
 // softmax arithmetic, not the tensor pipe, sets the pace of a key tile.
-int softmax_groups_for(int mode, int D) {
+int softmax_groups_for(int mode, int D, int tiles_per_item) {
     const int forced = g_tune_softmax_groups.load(std::memory_order_relaxed);
     if (forced == 1 || forced == 2) return forced;
-    (void)mode;
     // Measured on B200 (image- and video-length self-attention): at D = 64 the tensor work per key tile is half
-    // that of D = 128 while the softmax work is the same, and two groups are 1.1-1.3x faster in every mode; at
-    // D = 128 one group is as fast or faster (the tile period is set by the MMA-issuing warp there, which two
-    // more busy warps on its scheduler slow down).
-    return D == 64 ? 2 : 1;
+    // that of D = 128 while the softmax work is the same, and two groups are 1.1-1.3x faster in every mode.  At
+    // D = 128 the forward-only mode (a third of the tensor work of the JVP per tile) is 2-14 % faster with two
+    // groups from eight key tiles per item on; with tangents one group is as fast or faster.
+    if (D == 64) return 2;
+    return (mode == attn_jvp::kModeFwdOnly && tiles_per_item >= 8) ? 2 : 1;
 }
 
 int cuda_fail(const char* what, cudaError_t e) {
@@ -387,7 +387,7 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     }
     const long long n_ctas = (persistent && n_items > st.sm_count) ? st.sm_count : n_items;
     const dim3 grid((unsigned)n_ctas, 1, 1);
-    const int groups = softmax_groups_for(mode, D);
+    const int groups = softmax_groups_for(mode, D, tiles_per_item);
 #define ATTN_JVP_DISPATCH_G(DD, SS, GG)                                                                            \
     switch (mode) {                                                                                               \
         case attn_jvp::kModeJvp: rc = launch<DD, attn_jvp::kModeJvp, SS, GG>(maps, ka, grid, stream, st); break;   \

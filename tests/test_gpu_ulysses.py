@@ -35,6 +35,7 @@ def test_group_of_one_is_the_direct_call(aj):
     o2, to2, _ = layer(g["q"], g["k"], g["v"], g["tq"], kv_replicated=True)
     r2 = aj.attention_jvp(g["q"], g["k"], g["v"], g["tq"], None, None, scale=D ** -0.5)
     o3, to3, _ = layer(g["q"], g["k"], g["v"])
+    r3 = aj.attention_jvp(g["q"], g["k"], g["v"], None, None, None, scale=D ** -0.5, fwd_only=True)
     torch.cuda.synchronize()
     assert torch.equal(o2, r2[0]) and torch.equal(to2, r2[1])
-    assert to3 is None and torch.equal(o3, ro)
+    assert to3 is None and torch.equal(o3, r3[0])
