@@ -42,13 +42,16 @@ constexpr int kBlockN = 64;         // keys per tile (B_c)
 constexpr int kSoftmaxThreads = 128;   // four softmax warps per group: one thread per query row
 constexpr int kMmaWarp = 0;            // the two single-thread roles come first (oldest warps of the CTA)
 constexpr int kProducerWarp = 1;
-// One softmax group: warps 2..5 follow the two single-thread roles (192 threads).  Two groups (they take
-// alternate key tiles): the roles are laid out by warpgroup so that each can be given its own register budget --
-// warps 0..3 = MMA, producer and two idle warps, warps 4..7 = group 0, warps 8..11 = group 1 (384 threads).
-__host__ __device__ constexpr int first_softmax_warp(int groups) { return groups == 2 ? 4 : 2; }
-__host__ __device__ constexpr int num_threads(int groups) { return groups == 2 ? 384 : kSoftmaxThreads + 64; }
-constexpr int kRegsLightWarps = 104;    // two groups: registers per thread of warps 0..3 ...
-constexpr int kRegsSoftmaxWarps = 200; // ... and of the softmax warps (128 * 72 + 256 * 216 = 384 * 168)
+// The roles are laid out by warpgroup, so that each can be given its own register budget (384 threads):
+// warps 0..3 = MMA, producer and two idle warps; warps 4..7 = softmax group 0; warps 8..11 = softmax group 1 (two
+// groups take alternate key tiles), or, with one softmax group, the epilogue warps: they run the epilogue of every
+// work item (normalise, round, stage the output tiles), so that the softmax warps go straight on to the next item's
+// first key tile.  With two groups the group that finishes an item runs its epilogue while the other is already in
+// the next item.
+__host__ __device__ constexpr int first_softmax_warp(int) { return 4; }
+__host__ __device__ constexpr int num_threads(int) { return 3 * kSoftmaxThreads; }
+constexpr int kRegsLightWarps = 104;    // registers per thread of warps 0..3 ...
+constexpr int kRegsSoftmaxWarps = 200; // ... and of warps 4..11 (128 * 104 + 256 * 200 <= 384 * 168 = 64512)
 constexpr int kTmemCols = 512;
 constexpr int kScoreBufStride = 128; // tensor-memory columns of one score buffer {S 64, tS 64}
 constexpr float kRescaleThreshold = 8.0f;   // log2 units: rescale only when the max grows by > 2^8
@@ -131,7 +134,7 @@ struct SmemPlan {
     static constexpr int kQHalfBytes = kBlockM * 128;      // 16 KB: 128 rows x 128 B
     static constexpr int kQBytes = kHalves * kQHalfBytes;
     static constexpr int kKvHalfBytes = kBlockN * 128;     // 8 KB: 64 rows x 128 B
-    static constexpr bool kDoubleQ = !kPair && (MODE != kModeJvp || D == 64);
+    static constexpr bool kDoubleQ = kPair ? (MODE == kModeKvTangentFree) : (MODE != kModeJvp || D == 64);
     static constexpr int kQSets = kDoubleQ ? 2 : 1;
     static constexpr int kQSetBytes = (kDoubleQ && MODE == kModeFwdOnly) ? kQBytes : 2 * kQBytes;   // Q (+ tQ)
     static constexpr int kTilesPerSlot = (!kDoubleQ || MODE == kModeJvp) ? 2 : 1;                   // primal (+ tangent)
@@ -140,9 +143,10 @@ struct SmemPlan {
     static constexpr int kSlots = kDoubleQ ? (kRoom / kSlotBytes < 8 ? kRoom / kSlotBytes : 8) : ((D == 128) ? 5 : 8);
     static constexpr int kRingOffset = kQSets * kQSetBytes;
     static constexpr int kOperandBytes = kRingOffset + kSlots * kSlotBytes;
-    // Two softmax groups exchange four per-row fp32 values through shared memory (reference max, centring
-    // constant of tS, partial l and r), placed after the operand tiles.
-    static constexpr int kExchangeBytes = (kGroups == 2) ? 4 * kBlockM * 4 : 0;
+    // Four per-row fp32 values go through shared memory, placed after the operand tiles: two softmax groups exchange
+    // the reference max, the centring constant of tS and their partial l and r; with one group the softmax warps
+    // hand m, the centring constant, l and r of a finished item to the epilogue warps there.
+    static constexpr int kExchangeBytes = 4 * kBlockM * 4;
     // The dynamic allocation is declared 1024-byte aligned (the operand tiles need that for the 128-byte
     // swizzle); static shared memory (barriers, a few words) stays below 1 KB, so that at D = 128 operands
     // (224 KB), exchange area (2 KB) and static part fill the 227 KB a CTA can have exactly.
@@ -568,10 +572,10 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     __shared__ __align__(8) uint64_t bar_drain;
     __shared__ __align__(8) uint64_t bar_stage_ready;   // the item's staging slots are free of operand reads
     __shared__ __align__(8) uint64_t bar_stage_full;    // the softmax warps have written the item's output tiles
-    // two softmax groups, one barrier per quarter of the rows (a pair of warps, one of each group):
-    __shared__ __align__(8) uint64_t bar_m[4];          // the reference max after tile g is published (phase g & 1)
-    __shared__ __align__(8) uint64_t bar_fin[4];        // the non-finishing group's partial l, r of the item are published
-    __shared__ __align__(8) uint64_t bar_fin_read[4];   // ... and have been read by the finishing group
+    // one barrier per quarter of the rows (a pair of warps: one of each softmax group, or softmax and epilogue warp):
+    __shared__ __align__(8) uint64_t bar_m[4];          // two groups: the reference max after tile g is published (phase g & 1)
+    __shared__ __align__(8) uint64_t bar_fin[4];        // l, r (one group: also m, centring constant) of the item are published
+    __shared__ __align__(8) uint64_t bar_fin_read[4];   // ... and have been read by the warp that finishes the item
     __shared__ uint32_t tmem_base_smem;
     __shared__ int cta_abort;
 
@@ -748,10 +752,10 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     // shared-memory ring runs on without a break; per item it hands out 2 n slots to K/V tiles and then
     // kStageSlots slots to the output tiles.
 
-    // Two softmax groups: the warps of the first warpgroup need few registers (two of them are idle), the
-    // softmax warps hold a whole row of scores and tangent scores each; the budgets are moved accordingly.
+    // The warps of the first warpgroup need few registers (two of them are idle), the softmax warps hold a whole
+    // row of scores and tangent scores each; the budgets are moved accordingly.
     // (The forward-only softmax needs fewer registers than the 168 every thread of a 384-thread CTA starts with.)
-    constexpr bool kMoveRegs = (kGroups == 2) && kHasTQ;
+    constexpr bool kMoveRegs = kHasTQ;
     if (warp < kFirstSoftmaxWarp) {
     if (kMoveRegs) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLightWarps));
     if (warp == kProducerWarp) {
@@ -859,8 +863,22 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             int stage_slot[2] = {0, 0};
             int stage_it = 0;
             Item stage_w{};
-            auto store_staged = [&]() -> bool {
-                if (!mbar_wait(smem_u32(&bar_stage_full), stage_it & 1, abort_state)) return false;
+            // In two steps where the staging buffers are the item's Q/tQ buffers: the stores are issued as soon as the
+            // staged tiles are seen complete (`only_if_ready`: without waiting for them), and what needs their
+            // shared-memory reads to be over -- the load of the next item's Q, tQ into that buffer -- comes a tile
+            // later, so that this thread keeps the ring filled meanwhile instead of sitting in the wait.
+            bool stores_in_flight = false;
+            auto store_staged_finish = [&]() {
+                tma_store_wait_read();
+                TRACE(18, stage_it);  // producer: staging buffers read
+                stores_in_flight = false;
+            };
+            auto store_staged = [&](bool only_if_ready = false, bool finish = true) -> bool {
+                if (only_if_ready) {
+                    if (!mbar_test_wait(smem_u32(&bar_stage_full), stage_it & 1)) return true;
+                } else if (!mbar_wait(smem_u32(&bar_stage_full), stage_it & 1, abort_state)) {
+                    return false;
+                }
                 TRACE(17, stage_it);  // producer: staged tiles complete, stores issued next
                 // staged in two ring slots, or (two Q/tQ buffers) in the item's own Q and tQ buffer
                 const uint32_t src_o = kDoubleQ ? q_addr(stage_it) : smem_ring + stage_slot[0] * Plan::kSlotBytes;
@@ -873,11 +891,12 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                         tma_store_4d(&tm_to, src_t + hf * Plan::kQHalfBytes, hf * 64, stage_w.h, stage_w.q0, stage_w.b);
                 }
                 tma_store_commit();
+                stage_pending = false;
+                if (!finish) { stores_in_flight = true; return true; }
                 tma_store_wait_read();
                 // the slots go back to the ring (their `empty` phase is completed here instead of by an MMA commit)
                 for (int s = 0; s < kRingStage; ++s) mbar_arrive(smem_u32(&bar_slot_empty[stage_slot[s]]));
                 TRACE(18, stage_it);  // producer: staging slots back in the ring
-                stage_pending = false;
                 return true;
             };
             // hands the staging slots of item number `of_it` to the softmax warps; nothing is loaded into them, so
@@ -966,7 +985,16 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     }
                     if (ok) ok = load_v(j);
                     // the previous item's outputs: the loads above do not depend on its epilogue, the later ones do
-                    if (ok && (j == 1 || j + 1 == w.n_kv)) {
+                    // (Long enough items with two Q/tQ buffers: the stores go out at j = 1 or 2 if the staged tiles
+                    // are complete by then, at j = 3 at the latest; the next item's Q, tQ follow one tile after them.)
+                    constexpr bool kTwoStep = kPair && kDoubleQ && kStageSlots > 0;
+                    const bool two_step = kTwoStep && w.n_kv >= 6;
+                    if (two_step) {
+                        if (ok && stores_in_flight) store_staged_finish();          // (issued during the tile before)
+                        if (ok && stage_pending && j >= 1) ok = store_staged(j < 3, false);
+                    }
+                    if (ok && (two_step ? (!stage_pending && !stores_in_flight && j >= 1)
+                                        : (j == 1 || j + 1 == w.n_kv))) {
                         if (stage_pending) ok = store_staged();
                         if (kDoubleQ && ok && has_next && !next_q_loaded) {
                             // Two Q/tQ buffers: the other buffer held the item before and then its staged output
@@ -1278,6 +1306,10 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         // the epilogue while the other group is already in the next item.
         // =====================================================================================
         const int grp = (kGroups == 2) ? ((warp - kFirstSoftmaxWarp) >> 2) : 0;
+        // one group: warps 4..7 of this branch are the epilogue warps (same rows, i.e. tensor-memory lanes, as the
+        // softmax warp of their quarter)
+        constexpr bool kEpiWarps = (kGroups == 1);
+        const bool epi_role = kEpiWarps && (warp - kFirstSoftmaxWarp) >= 4;
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;                          // 0..127: a warp may only touch lanes 32*(warp%4)..+31
         const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
@@ -1317,7 +1349,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             // two groups: the group of the item's last tile finishes the item
             const bool finisher = (kGroups == 1) || (((g0 + n_kv - 1) & 1) == grp);
 
-            for (int j = 0; j < n_kv; ++j) {
+            for (int j = 0; j < (epi_role ? 0 : n_kv); ++j) {
                 const int g = g0 + j;
                 const int bsel = bp.buf;
                 const uint32_t bphase = bp.phase;
@@ -1539,6 +1571,30 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 continue;
             }
 
+            if (kEpiWarps) {
+                // One group: l, r, m and the centring constant of the finished item go to the epilogue warp of this
+                // quarter of the rows through the exchange words (single: the epilogue warp must have read the item
+                // before's), and the softmax warp goes on to the next item at once.
+                if (!epi_role) {
+                    if (it > 0 && !mbar_wait_warp(smem_u32(&bar_fin_read[quarter]), (it - 1) & 1, abort_state)) { ok = false; break; }
+                    st_shared_f32(xch_l, l_run);
+                    st_shared_f32(xch_r, r_run);
+                    st_shared_f32(xch_m, m_ref);
+                    st_shared_f32(xch_shift, ts_shift);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(finbar);
+                    g0 += n_kv;
+                    continue;
+                }
+                if (!mbar_wait_warp(finbar, it & 1, abort_state)) { ok = false; break; }
+                l_run = ld_shared_f32(xch_l);
+                r_run = ld_shared_f32(xch_r);
+                m_ref = ld_shared_f32(xch_m);
+                ts_shift = ld_shared_f32(xch_shift);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bar_fin_read[quarter]));
+            }
+
             // Epilogue: O/l, L = m + log l, tO = (T - r (O/l)) / l, once the item's last value MMAs are complete
             // (which implies all earlier ones).  A parity wait on bar_pv_done[g & 1] for tile g means what it should
             // only once the value MMAs of tile g - 2 (the barrier's previous phase) are known to be complete.  The
@@ -1590,59 +1646,113 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 stage_o = q_addr(it) + row * 128;
                 stage_t = tq_addr(it) + row * 128;
             }
+            if (kSplit || !kEpiWarps) {
+                // (two softmax groups: the epilogue shares its registers with the softmax pass, so it stays a rolled
+                // loop over 32-column chunks that stages each chunk at once)
 #pragma unroll 1
-            for (int c0 = 0; c0 < D; c0 += 32) {
-                uint32_t ov[32];
-                uint32_t tvv[32];
-                TMEM_LD32(tmem_o + lane_base + c0, ov, 0);
-                if (kHasTQ) TMEM_LD32(tmem_t + lane_base + c0, tvv, 0);
-                if (kRingStage > 0 && c0 == 0) {
-                    ok = mbar_wait_warp(smem_u32(&bar_stage_ready), it & 1, abort_state);
-                    if (!ok) { tc_wait_ld(); break; }
-                }
-                tc_wait_ld();
-                if (c0 + 32 >= D) {
-                    // O and T are in registers: the next item's first value MMA may overwrite them
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) arrive_at_issuer(smem_u32(&bar_acc_free));
-                }
-                if (kSplit) {
-#pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        const float o0 = __uint_as_float(ov[c]) * inv_l;
-                        ov[c] = __float_as_uint(o0);
-                        if (kHasTQ) tvv[c] = __float_as_uint(fmaf(-mu, o0, __uint_as_float(tvv[c]) * inv_l));
+                for (int c0 = 0; c0 < D; c0 += 32) {
+                    uint32_t ov[32];
+                    uint32_t tvv[32];
+                    TMEM_LD32(tmem_o + lane_base + c0, ov, 0);
+                    if (kHasTQ) TMEM_LD32(tmem_t + lane_base + c0, tvv, 0);
+                    if (!kSplit && kRingStage > 0 && c0 == 0) {
+                        ok = mbar_wait_warp(smem_u32(&bar_stage_ready), it & 1, abort_state);
+                        if (!ok) { tc_wait_ld(); break; }
                     }
-                    if (in_range) {
+                    tc_wait_ld();
+                    if (c0 + 32 >= D) {
+                        // O and T are in registers: the next item's first value MMA may overwrite them
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) arrive_at_issuer(smem_u32(&bar_acc_free));
+                    }
+                    if (kSplit) {
 #pragma unroll
-                        for (int v4 = 0; v4 < 8; ++v4) {
-                            *reinterpret_cast<uint4*>(po_row + c0 + v4 * 4) = make_uint4(ov[4 * v4], ov[4 * v4 + 1], ov[4 * v4 + 2], ov[4 * v4 + 3]);
-                            if (kHasTQ)
-                                *reinterpret_cast<uint4*>(pto_row + c0 + v4 * 4) = make_uint4(tvv[4 * v4], tvv[4 * v4 + 1], tvv[4 * v4 + 2], tvv[4 * v4 + 3]);
+                        for (int c = 0; c < 32; ++c) {
+                            const float o0 = __uint_as_float(ov[c]) * inv_l;
+                            ov[c] = __float_as_uint(o0);
+                            if (kHasTQ) tvv[c] = __float_as_uint(fmaf(-mu, o0, __uint_as_float(tvv[c]) * inv_l));
+                        }
+                        if (in_range) {
+#pragma unroll
+                            for (int v4 = 0; v4 < 8; ++v4) {
+                                *reinterpret_cast<uint4*>(po_row + c0 + v4 * 4) = make_uint4(ov[4 * v4], ov[4 * v4 + 1], ov[4 * v4 + 2], ov[4 * v4 + 3]);
+                                if (kHasTQ)
+                                    *reinterpret_cast<uint4*>(pto_row + c0 + v4 * 4) = make_uint4(tvv[4 * v4], tvv[4 * v4 + 1], tvv[4 * v4 + 2], tvv[4 * v4 + 3]);
+                            }
+                        }
+                    } else {
+                        uint32_t po[16], pt[16];
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            const float o0 = __uint_as_float(ov[2 * c]) * inv_l;
+                            const float o1 = __uint_as_float(ov[2 * c + 1]) * inv_l;
+                            po[c] = pack_bf16(o0, o1);
+                            if (kHasTQ) {
+                                const float t0 = fmaf(-mu, o0, __uint_as_float(tvv[2 * c]) * inv_l);
+                                const float t1 = fmaf(-mu, o1, __uint_as_float(tvv[2 * c + 1]) * inv_l);
+                                pt[c] = pack_bf16(t0, t1);
+                            }
+                        }
+                        // rows beyond Lq are staged too (the store clips them)
+                        const uint32_t half_off = (c0 >> 6) * Plan::kQHalfBytes;
+                        const int chunk0 = (c0 & 63) >> 3;
+#pragma unroll
+                        for (int v4 = 0; v4 < 4; ++v4) {
+                            const uint32_t off = half_off + (((chunk0 + v4) ^ (row & 7)) << 4);
+                            st_shared_v4(stage_o + off, po[4 * v4], po[4 * v4 + 1], po[4 * v4 + 2], po[4 * v4 + 3]);
+                            if (kHasTQ) st_shared_v4(stage_t + off, pt[4 * v4], pt[4 * v4 + 1], pt[4 * v4 + 2], pt[4 * v4 + 3]);
                         }
                     }
-                } else {
-                    uint32_t po[16], pt[16];
+                }
+            } else {
+                // The next item's first value MMAs wait for this: first everything that needs the accumulators (32
+                // columns of O and T at a time: load, normalise, round to bf16 and keep the packed row in registers),
+                // then the accumulators are given back, and only then is the row written to the staging buffer.
+                uint32_t po[D / 2];
+                uint32_t pt[kHasTQ ? D / 2 : 1];
+                const uint64_t inv2 = pack_f32x2(inv_l, inv_l);
+                const uint64_t negmu2 = pack_f32x2(-mu, -mu);
+#pragma unroll
+                for (int c0 = 0; c0 < D; c0 += 32) {
+                    uint32_t ov[32];
+                    uint32_t tvv[32];
+                    TMEM_LD32(tmem_o + lane_base + c0, ov, 0);
+                    if (kHasTQ) TMEM_LD32(tmem_t + lane_base + c0, tvv, 0);
+                    tc_wait_ld();
 #pragma unroll
                     for (int c = 0; c < 16; ++c) {
-                        const float o0 = __uint_as_float(ov[2 * c]) * inv_l;
-                        const float o1 = __uint_as_float(ov[2 * c + 1]) * inv_l;
-                        po[c] = pack_bf16(o0, o1);
+                        const uint64_t o2 = mul_f32x2(pack_f32x2(__uint_as_float(ov[2 * c]), __uint_as_float(ov[2 * c + 1])), inv2);
+                        float o0, o1;
+                        unpack_f32x2(o2, o0, o1);
+                        po[(c0 >> 1) + c] = pack_bf16(o0, o1);
                         if (kHasTQ) {
-                            const float t0 = fmaf(-mu, o0, __uint_as_float(tvv[2 * c]) * inv_l);
-                            const float t1 = fmaf(-mu, o1, __uint_as_float(tvv[2 * c + 1]) * inv_l);
-                            pt[c] = pack_bf16(t0, t1);
+                            const uint64_t tt = mul_f32x2(pack_f32x2(__uint_as_float(tvv[2 * c]), __uint_as_float(tvv[2 * c + 1])), inv2);
+                            float t0, t1;
+                            unpack_f32x2(fma_f32x2(negmu2, o2, tt), t0, t1);
+                            pt[(c0 >> 1) + c] = pack_bf16(t0, t1);
                         }
                     }
-                    // rows beyond Lq are staged too (the store clips them)
+                }
+                // O and T are in registers: the next item's first value MMA may overwrite them
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) arrive_at_issuer(smem_u32(&bar_acc_free));
+                if (kRingStage > 0) {
+                    ok = mbar_wait_warp(smem_u32(&bar_stage_ready), it & 1, abort_state);
+                    if (!ok) break;
+                }
+                // rows beyond Lq are staged too (the store clips them)
+#pragma unroll
+                for (int c0 = 0; c0 < D; c0 += 32) {
                     const uint32_t half_off = (c0 >> 6) * Plan::kQHalfBytes;
                     const int chunk0 = (c0 & 63) >> 3;
 #pragma unroll
                     for (int v4 = 0; v4 < 4; ++v4) {
                         const uint32_t off = half_off + (((chunk0 + v4) ^ (row & 7)) << 4);
-                        st_shared_v4(stage_o + off, po[4 * v4], po[4 * v4 + 1], po[4 * v4 + 2], po[4 * v4 + 3]);
-                        if (kHasTQ) st_shared_v4(stage_t + off, pt[4 * v4], pt[4 * v4 + 1], pt[4 * v4 + 2], pt[4 * v4 + 3]);
+                        const int q = (c0 >> 1) + 4 * v4;
+                        st_shared_v4(stage_o + off, po[q], po[q + 1], po[q + 2], po[q + 3]);
+                        if (kHasTQ) st_shared_v4(stage_t + off, pt[q], pt[q + 1], pt[q + 2], pt[q + 3]);
                     }
                 }
             }
@@ -1675,6 +1785,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         }
         if (warp == kFirstSoftmaxWarp + ((kMmaWarp - kFirstSoftmaxWarp) & 3)) {   // the softmax warp on the MMA warp's scheduler
             ACC_WRITE(2, acc_sm_scores);
+            if (!kEpiWarps) { ACC_WRITE(3, acc_sm_values); ACC_WRITE(4, acc_sm_epi); }
+        }
+        if (kEpiWarps && warp == kFirstSoftmaxWarp + 4 + ((kMmaWarp - kFirstSoftmaxWarp) & 3)) {   // ... and its epilogue warp
             ACC_WRITE(3, acc_sm_values);
             ACC_WRITE(4, acc_sm_epi);
         }
