@@ -43,8 +43,8 @@ DATASHEET_BF16_TFLOPS = 2250.0
 # head stay in L2 depends on the sequence length, so a workload takes the capture of its own class and scales it
 # by algorithmic bytes (within a class traffic is proportional to the tensors streamed once from HBM).
 NCU_TRAFFIC_BYTES = {
-    "short": {"workload": "image_dit_2b", "bytes": 254.2e6},     # L = 4096: 205.0 MB read + 49.2 MB written (two launches)
-    "long": {"workload": "video_dit_1p3b", "bytes": 940.7e6},    # L = 32760: 744.6 MB read + 196.1 MB written (one launch)
+    "short": {"workload": "image_dit_2b", "bytes": 256.0e6},     # L = 4096: 204.4 MB read + 51.6 MB written (two launches)
+    "long": {"workload": "video_dit_1p3b", "bytes": 1030.5e6},   # L = 32760: 820.1 MB read + 210.4 MB written (one launch)
 }
 
 
