@@ -202,11 +202,12 @@ int attn_jvp_fwd_splitkv_static(const void* q, const void* k, const void* v,
 /*
  * Tuning knobs for benchmarking and A/B comparisons (process-wide; the paper has no counterpart).  Every setting
  * computes the same function within the library's tolerance; only the kernel variant changes.
- *   ATTN_JVP_TUNE_SOFTMAX_GROUPS  0 = the library chooses per (mode, D) (default), 1 = one softmax warpgroup per
- *                                 CTA (192 threads), 2 = two warpgroups taking alternate key tiles (384 threads).
- *   ATTN_JVP_TUNE_CTA_PAIR        0 = the library chooses (default), 1 = never, 2 = whenever it exists (full JVP,
- *                                 D = 128, no key chunks): the kernel variant in which two CTAs on neighbouring SMs
- *                                 share a 256-row query block, the K/V operand tiles and one MMA instruction stream.
+ *   ATTN_JVP_TUNE_SOFTMAX_GROUPS  0 = the library chooses per (mode, D, keys) (default), 1 = one softmax warpgroup
+ *                                 per CTA plus a warpgroup that runs the work items' epilogues, 2 = two softmax
+ *                                 warpgroups taking alternate key tiles (384 threads either way).
+ *   ATTN_JVP_TUNE_CTA_PAIR        0 = the library chooses (default), 1 = never, 2 = whenever it exists (D = 128, no
+ *                                 key chunks): the kernel variant in which two CTAs on neighbouring SMs share a
+ *                                 256-row query block, the K/V operand tiles and one MMA instruction stream.
  * Returns 0, or ATTN_JVP_ERR_FLAGS for an unknown knob or value.
  */
 #define ATTN_JVP_TUNE_SOFTMAX_GROUPS 1

@@ -2,15 +2,17 @@
 //
 // One CTA owns a 128-row query tile of one (batch, head) and streams the keys in
 // tiles of 64; CTAs are persistent (one per SM) and walk the query tiles round-robin, so that the epilogue of
-// one tile overlaps the loads and the first score MMAs of the next.  Roles (warp-specialised, 192 threads):
-//   warp 0     MMA issuer: the whole warp runs the loop in lock step, one elected lane issues
-//              tcgen05.mma with accumulators in tensor memory.
-//   warp 1     TMA producer: Q,tQ per query tile, K|tK and V|tV tiles into a shared-memory ring.
-//   warps 2-5  softmax: thread (w, lane) owns query row 32*(w%4) + lane (its tensor-memory lane) and
-//              all 64 columns of every score tile.  Reads S and tS from tensor memory, keeps m, l, r
-//              (Algorithm 2 lines 10-12, 16) in registers, writes P~ and H~ = P~ . tS back to tensor
-//              memory as bf16 MMA operands, rescales the accumulators when the running max moves, and
-//              runs the epilogue (lines 19-23).
+// one tile overlaps the loads and the first score MMAs of the next.  Roles (warp-specialised, 384 threads, laid
+// out by warpgroup so that each can have its own register budget):
+//   warp 0      MMA issuer: the whole warp runs the loop in lock step, one elected lane's tcgen05.mma take effect,
+//               with accumulators in tensor memory.
+//   warp 1      TMA producer: Q,tQ per query tile, K|tK and V|tV tiles into a shared-memory ring.  (Warps 2, 3 idle.)
+//   warps 4-7   softmax: thread (w, lane) owns query row 32*(w%4) + lane (its tensor-memory lane) and
+//               all 64 columns of every score tile.  Reads S and tS from tensor memory, keeps m, l, r
+//               (Algorithm 2 lines 10-12, 16) in registers, writes P~ and H~ = P~ . tS back to tensor
+//               memory as bf16 MMA operands, and rescales the accumulators when the running max moves.
+//   warps 8-11  a second softmax group on alternate key tiles, or (one group) the epilogue warps, which run
+//               lines 19-23 for every finished query tile while the softmax warps are in the next one.
 //
 // Tensor-memory map (512 columns x 128 lanes, fp32):
 //   [0, D)        O  accumulator (line 13)

@@ -3,10 +3,13 @@
 Builds a second copy of the library with -DATTN_JVP_TRACE=2 (clock64 stamps at the hand-over points of the
 roles of one CTA, see attn_jvp_kernel.cuh), runs one shape through it and prints, per 64-key tile, when the MMA
 warp issued the score and value MMAs and when the softmax warps saw the scores, agreed on the reference max,
-stored P~ and handed the tile back -- plus the mean tile period.  The cycle figures quoted in the design doc and
-profiles/ come from this tool:
+stored P~ and handed the tile back -- plus the mean tile period:
 
     python -m paper_2510_08431_b200.trace --B 1 --H 8 --Lq 18944 --Lk 4096 --D 128 [--mode jvp|kv_free|fwd] [--groups 1|2] [--pair 1|2]
+
+With --totals the build is -DATTN_JVP_TRACE=1 instead: no per-tile stamps (they cost the MMA warp 10-20 % of a
+tile), only the cycles each role of the traced CTA spent in blocking waits, summed in a register and written once
+at the end -- who waits for whom, at the shipped build's speed.
 """
 from __future__ import annotations
 
@@ -23,22 +26,24 @@ from . import build as lib_build
 from . import synth
 
 TRACE_LIB = os.path.join(lib_build.PKG, "libattn_jvp_trace.so")
+TOTALS_LIB = os.path.join(lib_build.PKG, "libattn_jvp_trace_totals.so")
 EVENTS, STEPS = 32, 96
 
 
-def build_trace_library() -> str:
-    stale = (not os.path.exists(TRACE_LIB)) or any(os.path.getmtime(d) > os.path.getmtime(TRACE_LIB) for d in lib_build.DEPS)
+def build_trace_library(level: int = 2) -> str:
+    path = TRACE_LIB if level == 2 else TOTALS_LIB
+    stale = (not os.path.exists(path)) or any(os.path.getmtime(d) > os.path.getmtime(path) for d in lib_build.DEPS)
     if stale:
         cmd = [lib_build._nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-               "-DATTN_JVP_TRACE=2", "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(lib_build.ROOT, "include"),
-               "-o", TRACE_LIB, lib_build.SRC, "-lcudart"]
+               f"-DATTN_JVP_TRACE={level}", "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(lib_build.ROOT, "include"),
+               "-o", path, lib_build.SRC, "-lcudart"]
         subprocess.run(cmd, check=True, capture_output=True)
-    return TRACE_LIB
+    return path
 
 
-def run(B, H, Lq, Lk, D, mode="jvp", groups=0, first=20, count=6, seed=4, pair=0):
+def run(B, H, Lq, Lk, D, mode="jvp", groups=0, first=20, count=6, seed=4, pair=0, level=2):
     """Runs the shape three times through the trace build and returns the [EVENTS][STEPS] stamp array."""
-    lib = ctypes.CDLL(build_trace_library())
+    lib = ctypes.CDLL(build_trace_library(level))
     x = synth.make_inputs(B, H, Lq, Lk, D, 1.0, 0.5, seed, kv_tangent_free=(mode != "jvp"))
     g = {k: (None if t is None else t.cuda()) for k, t in x.items()}
     flags = {"jvp": 0, "kv_free": binding.KV_TANGENT_FREE, "fwd": binding.FWD_ONLY}[mode]
@@ -104,6 +109,23 @@ def report(t, first=20, count=6):
           int(t[EVENTS - 1][1] - t[EVENTS - 1][0]), "cycles")
 
 
+TOTALS = ["MMA warp blocked for a tile's P~ / operands", "MMA warp blocked at an item's start",
+          "softmax warp blocked for the next scores", "epilogue: blocked for the item's last value MMAs",
+          "epilogue: its own run"]
+
+
+def report_totals(t, Lk):
+    """Blocked-cycle totals of the traced CTA's roles (level-1 build): row EVENTS - 2 holds (cycles, count) pairs."""
+    life = int(t[EVENTS - 1][1] - t[EVENTS - 1][0])
+    tiles = int(t[EVENTS - 2][5])          # the softmax warp waits once per key tile
+    n_kv = (Lk + 63) // 64
+    print(f"CTA lifetime {life} cycles, {tiles} key tiles, {tiles / n_kv:.1f} work items: "
+          f"{life / max(tiles, 1):.0f} cycles per tile, {life * n_kv / max(tiles, 1):.0f} per item")
+    for k, name in enumerate(TOTALS):
+        tot, n = int(t[EVENTS - 2][2 * k]), int(t[EVENTS - 2][2 * k + 1])
+        print(f"  {name:50s} {tot:9d} cycles = {100.0 * tot / life:5.1f} % of the lifetime, {n} times, mean {tot / max(n, 1):.0f}")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--B", type=int, default=1); ap.add_argument("--H", type=int, default=8)
@@ -114,7 +136,11 @@ def main():
     ap.add_argument("--pair", type=int, default=0, help="CTA-pair kernel: 0 library's choice, 1 off, 2 on")
     ap.add_argument("--first", type=int, default=20); ap.add_argument("--count", type=int, default=4)
     ap.add_argument("--items", action="store_true", help="print the hand-over between work items instead of the tiles")
+    ap.add_argument("--totals", action="store_true", help="blocked-cycle totals per role (no per-tile stamps)")
     a = ap.parse_args()
+    if a.totals:
+        report_totals(run(a.B, a.H, a.Lq, a.Lk, a.D, a.mode, a.groups, pair=a.pair, level=1), a.Lk)
+        return
     t = run(a.B, a.H, a.Lq, a.Lk, a.D, a.mode, a.groups, pair=a.pair)
     if a.items:
         report_items(t, tiles_per_item=(a.Lk + 63) // 64)
