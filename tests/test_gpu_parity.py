@@ -121,9 +121,11 @@ def _rel_l2_only(oracle, x, B, H, Lq, Lk, D, scale, o, to, lse):
     assert np.abs(gL - rL).max() <= 1e-3 * (1 + np.abs(rL).max())
 
 
+@pytest.mark.parametrize("D,Lk", [(64, 200), (128, 520)])
 @pytest.mark.parametrize("scale", [-0.2, 0.0, 1.0])
-def test_unusual_scales(aj, oracle, scale):
-    B, H, Lq, Lk, D = 1, 2, 130, 200, 64
+def test_unusual_scales(aj, oracle, scale, D, Lk):
+    """Negative, zero (keys past Lk must still drop out: the last key tile is ragged) and large scales."""
+    B, H, Lq = 1, 2, 130
     x = synth.make_inputs(B, H, Lq, Lk, D, 0.7, 0.5, seed=45)
     o, to, lse = U.run(aj, U.to_gpu(x), scale)
     if scale == 1.0:   # score std ~ 4: peaked softmax

@@ -1,6 +1,6 @@
 """Persistent CTAs: several work items per CTA with very few key tiles each.
 
-With one to six 64-key tiles per item the hand-over between items (shared-memory ring running on across items,
+With one to nine 64-key tiles per item the hand-over between items (shared-memory ring running on across items,
 staging slots for the output tiles interleaved with the next item's loads, reuse of the accumulators) makes up
 most of what a CTA does, and every ring position is reused after a different predecessor than in long items.
 Every item is checked against the fp64 oracle on a few of its rows.
@@ -35,7 +35,7 @@ def _rows_touching_every_item(B, H, Lq, stride=37):
 
 @pytest.mark.parametrize("D", [64, 128])
 @pytest.mark.parametrize("mode", ["jvp", "kv_free", "fwd"])
-@pytest.mark.parametrize("n_tiles", [1, 2, 3, 4, 6])
+@pytest.mark.parametrize("n_tiles", [1, 2, 3, 4, 6, 8, 9])
 def test_many_short_items_per_cta(aj, oracle, D, mode, n_tiles):
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     B, H = 1, 3
