@@ -141,9 +141,10 @@ int attn_jvp_fwd_splitkv(const void* q, const void* k, const void* v,
  * next group in and the previous group out.  Every (b, h) is computed exactly as by attn_jvp_fwd on a device
  * tensor (the result of a head does not depend on the other heads), so the outputs are bit-identical.
  *
- *   heads_per_stage  heads per pipeline stage; 0 = library default (about five stages, copy rows >= 512 bytes).
+ *   heads_per_stage  heads per pipeline stage; 0 = library default (about ten stages where the kernel takes as
+ *                    long as the copies, about five where the copies set the pace; copy rows >= 512 bytes).
  *   workspace        DEVICE scratch owned by the caller, 256-byte aligned, at least
- *                    attn_jvp_host_workspace_bytes(...) bytes (two buffer sets of one head group: eight bf16
+ *                    attn_jvp_host_workspace_bytes(...) bytes (three buffer sets of one head group: eight bf16
  *                    tensors and the LSE block); contents undefined afterwards.  Two calls that share a
  *                    workspace must be ordered on the GPU (same stream, or an event between their streams).
  *   cuda_stream      the work is ordered after what is already on this stream, and the stream continues only

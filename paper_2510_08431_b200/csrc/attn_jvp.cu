@@ -425,11 +425,14 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
 // Host-buffer pipeline: the heads are processed in groups; while the kernel works on one group, the copy
 // engines bring in the next group's inputs and take out the previous group's outputs.
 // ---------------------------------------------------------------------------------------------
+// Buffer sets of the host pipeline: with three, the copy-in of group g + 2 no longer waits for the copy-out of
+// group g (with two sets a stage took copy-in + copy-out, 10.7 ms on the headline shape, instead of the kernel's 9.2).
+constexpr int kHostSets = 3;
 struct HostPipe {
     bool ready = false;
     cudaStream_t in = nullptr, comp = nullptr, out = nullptr;
-    cudaEvent_t start = nullptr, in_done[2] = {}, comp_done[2] = {}, out_done[2] = {}, end_in = nullptr,
-                end_comp = nullptr, end_out = nullptr;
+    cudaEvent_t start = nullptr, in_done[kHostSets] = {}, comp_done[kHostSets] = {}, out_done[kHostSets] = {},
+                end_in = nullptr, end_comp = nullptr, end_out = nullptr;
     std::mutex lock;     // one enqueue at a time per device: the events are reused from call to call
 };
 HostPipe g_host_pipe[kMaxDevices];
@@ -438,8 +441,12 @@ HostPipe g_host_pipe[kMaxDevices];
 int host_pipe_setup(HostPipe& hp) {
     if (hp.ready) return 0;
     cudaStream_t* streams[3] = {&hp.in, &hp.comp, &hp.out};
-    cudaEvent_t* events[10] = {&hp.start, &hp.in_done[0], &hp.in_done[1], &hp.comp_done[0], &hp.comp_done[1],
-                               &hp.out_done[0], &hp.out_done[1], &hp.end_in, &hp.end_comp, &hp.end_out};
+    cudaEvent_t* events[4 + 3 * kHostSets] = {&hp.start, &hp.end_in, &hp.end_comp, &hp.end_out};
+    for (int i = 0; i < kHostSets; ++i) {
+        events[4 + 3 * i] = &hp.in_done[i];
+        events[5 + 3 * i] = &hp.comp_done[i];
+        events[6 + 3 * i] = &hp.out_done[i];
+    }
     cudaError_t e = cudaSuccess;
     const char* what = nullptr;
     for (cudaStream_t* st : streams) {
@@ -461,10 +468,20 @@ int host_pipe_setup(HostPipe& hp) {
     return 0;
 }
 
-// Heads per pipeline stage: the caller's choice, else about five stages, with copy rows of at least 512 bytes.
-int host_heads_per_stage(int H, int D, int requested) {
+// Heads per pipeline stage: the caller's choice; else about ten stages where the kernel takes about as long as the
+// copies or longer (the first group's copy-in and the last group's copy-out are not overlapped with anything, so
+// short stages pay), and about five where the copies set the pace (their rows get longer, which the copy engines
+// like: measured 16.4 against 18.6 ms on the 512-key cross-attention shape); copy rows of at least 512 bytes.
+int host_heads_per_stage(int B, int H, int Lq, int Lk, int D, unsigned flags, int requested) {
     if (requested > 0) return requested < H ? requested : H;
-    int hg = (H + 4) / 5;
+    const bool fwd_only = (flags & ATTN_JVP_FWD_ONLY) != 0;
+    const bool jvp_kv = !fwd_only && (flags & ATTN_JVP_KV_TANGENT_FREE) == 0;
+    const double cells = (double)B * H * (double)Lq * (double)Lk * D;
+    const double t_kernel = (fwd_only ? 4.0 : (jvp_kv ? 12.0 : 8.0)) * cells / 1.3e15;           // seconds, roughly
+    const double bytes_in = 2.0 * D * B * H * ((fwd_only ? 1.0 : 2.0) * Lq + (jvp_kv ? 4.0 : 2.0) * Lk);
+    const double t_copy = bytes_in / 45e9;
+    const int stages = (t_kernel > 0.8 * t_copy) ? 10 : 5;
+    int hg = (H + stages - 1) / stages;
     const int min_heads = (512 + D * 2 - 1) / (D * 2);
     if (hg < min_heads) hg = min_heads;
     return hg < H ? hg : H;
@@ -473,7 +490,7 @@ int host_heads_per_stage(int H, int D, int requested) {
 struct HostLayout {
     size_t nq, nk, nl;     // bytes of one Q-side tensor, one K-side tensor, the LSE block of a head group (padded)
     size_t set_bytes;      // one buffer set: q, tq, o, to, k, v, tk, tv, lse
-    size_t total;          // two sets
+    size_t total;          // kHostSets sets
 };
 HostLayout host_layout(int B, int Lq, int Lk, int D, int hg) {
     auto pad = [](size_t n) { return (n + 255) & ~(size_t)255; };
@@ -482,7 +499,7 @@ HostLayout host_layout(int B, int Lq, int Lk, int D, int hg) {
     L.nk = pad((size_t)B * Lk * hg * D * 2);
     L.nl = pad((size_t)B * hg * Lq * 4);
     L.set_bytes = 4 * L.nq + 4 * L.nk + L.nl;
-    L.total = 2 * L.set_bytes;
+    L.total = kHostSets * L.set_bytes;
     return L;
 }
 
@@ -501,7 +518,7 @@ int run_host(const void* q, const void* k, const void* v, const void* tq, const 
     if (jvp_kv && (!tk || !tv)) return ATTN_JVP_ERR_NULL;
     if (!std::isfinite(scale)) return ATTN_JVP_ERR_SCALE;
     if ((uintptr_t)workspace & 255u) return ATTN_JVP_ERR_ALIGN;
-    const int hg = host_heads_per_stage(H, D, heads_per_stage);
+    const int hg = host_heads_per_stage(B, H, Lq, Lk, D, flags, heads_per_stage);
     const HostLayout lay = host_layout(B, Lq, Lk, D, hg);
     if (workspace_bytes < lay.total) return ATTN_JVP_ERR_WORKSPACE;
 
@@ -529,7 +546,7 @@ int run_host(const void* q, const void* k, const void* v, const void* tq, const 
 
     const int n_stages = (H + hg - 1) / hg;
     for (int g = 0; g < n_stages && rc == 0 && ce == cudaSuccess; ++g) {
-        const int set = g & 1;
+        const int set = g % kHostSets;
         const int h0 = g * hg;
         const int hc = (H - h0 < hg) ? H - h0 : hg;
         char* base = static_cast<char*>(workspace) + (size_t)set * lay.set_bytes;
@@ -546,7 +563,7 @@ int run_host(const void* q, const void* k, const void* v, const void* tq, const 
         const size_t head_off = (size_t)h0 * D * 2;
 
         // inputs of this group: gather the group's heads out of the interleaved host rows
-        if (g >= 2) check(cudaStreamWaitEvent(hp.in, hp.out_done[set], 0), "cudaStreamWaitEvent");
+        if (g >= kHostSets) check(cudaStreamWaitEvent(hp.in, hp.out_done[set], 0), "cudaStreamWaitEvent");
         auto h2d = [&](char* dst, const void* src, int L) {
             check(cudaMemcpy2DAsync(dst, row_dev, static_cast<const char*>(src) + head_off, row_host, row_dev,
                                     (size_t)B * L, cudaMemcpyHostToDevice, hp.in), "cudaMemcpy2DAsync (host to device)");
@@ -653,7 +670,11 @@ int attn_jvp_fwd_splitkv(const void* q, const void* k, const void* v, const void
 
 size_t attn_jvp_host_workspace_bytes(int B, int H, int Lq, int Lk, int D, int heads_per_stage) {
     if (B < 1 || H < 1 || Lq < 1 || Lk < 1 || (D != 64 && D != 128) || heads_per_stage < 0) return 0;
-    return host_layout(B, Lq, Lk, D, host_heads_per_stage(H, D, heads_per_stage)).total;
+    // (the default stage length depends on the flags, which this function does not get: the size covers the longer
+    // of the two, five stages' worth of heads, which both flag-dependent choices fit into)
+    const int hg_copy_bound = host_heads_per_stage(B, H, Lq, 1, D, ATTN_JVP_FWD_ONLY, heads_per_stage);
+    const int hg_here = host_heads_per_stage(B, H, Lq, Lk, D, 0u, heads_per_stage);
+    return host_layout(B, Lq, Lk, D, hg_copy_bound > hg_here ? hg_copy_bound : hg_here).total;
 }
 
 int attn_jvp_fwd_host(const void* q, const void* k, const void* v, const void* tq, const void* tk, const void* tv,

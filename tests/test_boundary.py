@@ -129,12 +129,12 @@ def test_workspace_size_functions_are_plain_host_arithmetic(lib):
     four = lib.attn_jvp_splitkv_workspace_bytes(B, H, Lq, Lk, D, 4)
     assert four == 2 * 4 * B * Lq * H * D * 4 + 2 * 4 * B * H * Lq * 4
     assert lib.attn_jvp_splitkv_workspace_bytes(B, H, Lq, Lk, 96, 4) == 0
-    # host pipeline: two buffer sets of one head group (4 Q-side + 4 K-side bf16 tensors + LSE, 256-byte padded)
+    # host pipeline: three buffer sets of one head group (default: sized for five stages' worth of heads) (4 Q-side + 4 K-side bf16 tensors + LSE, 256-byte padded)
     pad = lambda n: (n + 255) // 256 * 256
     for (B, H, Lq, Lk, D, hps, hg) in ((1, 40, 32760, 32760, 128, 0, 8), (1, 40, 32760, 32760, 128, 3, 3),
                                        (2, 5, 300, 200, 128, 2, 2), (1, 7, 129, 513, 64, 0, 4),
                                        (1, 3, 50, 60, 64, 0, 3), (1, 2, 50, 60, 128, 9, 2)):
-        want = 2 * (4 * pad(B * Lq * hg * D * 2) + 4 * pad(B * Lk * hg * D * 2) + pad(B * hg * Lq * 4))
+        want = 3 * (4 * pad(B * Lq * hg * D * 2) + 4 * pad(B * Lk * hg * D * 2) + pad(B * hg * Lq * 4))
         assert lib.attn_jvp_host_workspace_bytes(B, H, Lq, Lk, D, hps) == want
     assert lib.attn_jvp_host_workspace_bytes(1, 4, 64, 64, 96, 0) == 0
     assert lib.attn_jvp_host_workspace_bytes(1, 4, 64, 64, 64, -1) == 0
