@@ -544,11 +544,15 @@ int run_host(const void* q, const void* k, const void* v, const void* tq, const 
     cudaStream_t internal[3] = {hp.in, hp.comp, hp.out};
     for (cudaStream_t st : internal) check(cudaStreamWaitEvent(st, hp.start, 0), "cudaStreamWaitEvent");
 
-    const int n_stages = (H + hg - 1) / hg;
-    for (int g = 0; g < n_stages && rc == 0 && ce == cudaSuccess; ++g) {
+    // The first group's copy-in and the last group's copy-out overlap with nothing: with enough groups the first one
+    // is half as long, which (for a head count that is a multiple of the group length) leaves a short one at the
+    // end as well.
+    const int first_hc = (hg >= 2 && H >= 4 * hg) ? hg / 2 : hg;
+    int h0 = 0;
+    for (int g = 0; h0 < H && rc == 0 && ce == cudaSuccess; ++g) {
         const int set = g % kHostSets;
-        const int h0 = g * hg;
-        const int hc = (H - h0 < hg) ? H - h0 : hg;
+        const int want = (g == 0) ? first_hc : hg;
+        const int hc = (H - h0 < want) ? H - h0 : want;
         char* base = static_cast<char*>(workspace) + (size_t)set * lay.set_bytes;
         char* d_q = base;
         char* d_tq = d_q + lay.nq;
@@ -596,6 +600,7 @@ int run_host(const void* q, const void* k, const void* v, const void* tq, const 
                                 (size_t)hc * Lq * 4, (size_t)B, cudaMemcpyDeviceToHost, hp.out),
               "cudaMemcpy2DAsync (LSE)");
         check(cudaEventRecord(hp.out_done[set], hp.out), "cudaEventRecord");
+        h0 += hc;
     }
     // ... and the caller's stream continues after all of it (also when an error cut the loop short: the internal
     // streams are never left chained to the caller's stream without the closing join)
