@@ -180,7 +180,7 @@ bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
 template <int D, int MODE, bool SPLIT, int GROUPS, bool PAIR = false>
 int launch(const CUtensorMap* maps, const KernelArgs& ka, dim3 grid, cudaStream_t stream, DeviceState& st) {
     auto kern = attn_jvp::attn_jvp_fwd_kernel<D, MODE, SPLIT, GROUPS, PAIR>;
-    using Plan = attn_jvp::SmemPlan<D, MODE, GROUPS, PAIR>;
+    using Plan = attn_jvp::SmemPlan<D, MODE, GROUPS, PAIR, SPLIT>;
     std::atomic<int>& slot = PAIR ? st.dyn_smem_pair[MODE][GROUPS - 1] : st.dyn_smem[D == 128][MODE][SPLIT][GROUPS - 1];
     int smem = slot.load(std::memory_order_acquire);
     if (smem == 0) {
@@ -311,14 +311,20 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     }
     cudaError_t e;
 
-    // ---- tensor maps (Q-side boxes are 128 rows, K-side boxes 64 rows) ----
+    // ---- which kernel variant (decided on the number of 64-key tiles per item), and its key-tile size ----
+    const int tiles64 = (Lk + attn_jvp::kBlockN - 1) / attn_jvp::kBlockN;
+    const int tiles_per_item = split ? tiles_per_split : tiles64;
+    const bool pair = use_cta_pair(mode, D, split, tiles_per_item);
+    const int key_tile = attn_jvp::key_tile(D, mode, split, pair);
+
+    // ---- tensor maps (Q-side boxes are 128 rows, K-side boxes one key tile) ----
     CUtensorMap maps[9];
     if (int rc = make_map(&maps[0], q, B, Lq, H, D, attn_jvp::kBlockM)) return rc;
-    if (int rc = make_map(&maps[1], k, B, Lk, H, D, attn_jvp::kBlockN)) return rc;
-    if (int rc = make_map(&maps[2], v, B, Lk, H, D, attn_jvp::kBlockN)) return rc;
+    if (int rc = make_map(&maps[1], k, B, Lk, H, D, key_tile)) return rc;
+    if (int rc = make_map(&maps[2], v, B, Lk, H, D, key_tile)) return rc;
     if (int rc = make_map(&maps[3], fwd_only ? q : tq, B, Lq, H, D, attn_jvp::kBlockM)) return rc;
-    if (int rc = make_map(&maps[4], mode == attn_jvp::kModeJvp ? tk : k, B, Lk, H, D, attn_jvp::kBlockN)) return rc;
-    if (int rc = make_map(&maps[5], mode == attn_jvp::kModeJvp ? tv : v, B, Lk, H, D, attn_jvp::kBlockN)) return rc;
+    if (int rc = make_map(&maps[4], mode == attn_jvp::kModeJvp ? tk : k, B, Lk, H, D, key_tile)) return rc;
+    if (int rc = make_map(&maps[5], mode == attn_jvp::kModeJvp ? tv : v, B, Lk, H, D, key_tile)) return rc;
     // output tiles (bf16, stored from shared memory by TMA; the split-KV kernel does not use these two)
     if (int rc = make_map(&maps[6], o, B, Lq, H, D, attn_jvp::kBlockM)) return rc;
     if (int rc = make_map(&maps[7], fwd_only ? o : to, B, Lq, H, D, attn_jvp::kBlockM)) return rc;
@@ -335,7 +341,7 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     ka.H = H;
     ka.Lq = Lq;
     ka.Lk = Lk;
-    ka.n_kv_tiles = (Lk + attn_jvp::kBlockN - 1) / attn_jvp::kBlockN;
+    ka.n_kv_tiles = (Lk + key_tile - 1) / key_tile;
     ka.scale = scale;
     // The kernel masks the keys past Lk by setting their scaled score to -inf, which needs a nonzero factor: a zero
     // scale (every score 0) is computed with 2^-100 in the exponent, which changes no result bit (tS keeps the 0).
@@ -359,10 +365,9 @@ int run(const void* q, const void* k, const void* v, const void* tq, const void*
     // Short items (few key tiles): one persistent CTA per SM, so that the epilogue of an item overlaps the
     // start of the next.  Long items: one CTA per item, which lets the hardware balance the load (a static
     // round-robin costs up to one item of imbalance at the end, which is more than the overlap saves there).
-    const int tiles_per_item = split ? tiles_per_split : ka.n_kv_tiles;
     const bool persistent = tiles_per_item <= kPersistentMaxTiles;
     int rc;
-    if (use_cta_pair(mode, D, split, tiles_per_item)) {
+    if (pair) {
         // A work item is a 256-row query block (two tiles, one per CTA of a pair); with an odd number of tiles the
         // last pair's second CTA has no rows and writes nothing.
         const long long n_q_pairs = (n_q_tiles + 1) / 2;

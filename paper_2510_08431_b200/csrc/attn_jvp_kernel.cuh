@@ -40,7 +40,7 @@
 namespace attn_jvp {
 
 constexpr int kBlockM = 128;        // query rows per CTA (B_r)
-constexpr int kBlockN = 64;         // keys per tile (B_c)
+constexpr int kBlockN = 64;         // keys per tile (B_c) ...
 constexpr int kSoftmaxThreads = 128;   // four softmax warps per group: one thread per query row
 constexpr int kMmaWarp = 0;            // the two single-thread roles come first (oldest warps of the CTA)
 constexpr int kProducerWarp = 1;
@@ -130,12 +130,21 @@ struct KernelArgs {
 //   Two Q/tQ buffers (the variants that leave room: no K/V tangents, or D = 64): the next item's Q, tQ are loaded
 //   while the current item runs, ring slots hold exactly what the mode loads, and an item's output tiles are staged
 //   in its own Q/tQ buffer (dead once its last value MMAs are complete) instead of in ring slots.
-template <int D, int MODE, int kGroups, bool kPair>
+// ... except in the forward-only mode at D = 128 (one CTA per query tile, no key chunks), which takes 128 keys per
+// tile: there is no tS, so a score buffer of 128 tensor-memory columns holds S of 128 keys, the N = 128 score MMAs
+// run at the pipe's full rate (64 cycles for twice the work of an N = 64 one at 54), and the per-tile costs of
+// the issuing and softmax warps (barriers, tensor-memory round trips, bookkeeping) are paid half as often.
+__host__ __device__ constexpr int key_tile(int D, int mode, bool split, bool pair) {
+    return (mode == kModeFwdOnly && D == 128 && !split && !pair) ? 2 * kBlockN : kBlockN;
+}
+
+template <int D, int MODE, int kGroups, bool kPair, bool kSplit = false>
 struct SmemPlan {
+    static constexpr int kBN = key_tile(D, MODE, kSplit, kPair);   // keys per tile
     static constexpr int kHalves = D / 64;                 // 64-element (128-byte) swizzle atoms per row
     static constexpr int kQHalfBytes = kBlockM * 128;      // 16 KB: 128 rows x 128 B
     static constexpr int kQBytes = kHalves * kQHalfBytes;
-    static constexpr int kKvHalfBytes = kBlockN * 128;     // 8 KB: 64 rows x 128 B
+    static constexpr int kKvHalfBytes = kBN * 128;         // 8 KB: 64 rows x 128 B (16 KB with 128-key tiles)
     static constexpr bool kDoubleQ = kPair ? (MODE == kModeKvTangentFree) : (MODE != kModeJvp || D == 64);
     static constexpr int kQSets = kDoubleQ ? 2 : 1;
     static constexpr int kQSetBytes = (kDoubleQ && MODE == kModeFwdOnly) ? kQBytes : 2 * kQBytes;   // Q (+ tQ)
@@ -542,7 +551,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     const __grid_constant__ CUtensorMap tm_o, const __grid_constant__ CUtensorMap tm_to,
                     const __grid_constant__ CUtensorMap tm_k32, const KernelArgs args) {
     static_assert(!kPair || (D == 128 && !kSplit), "the CTA-pair variant exists at D = 128, without key chunks");
-    using Plan = SmemPlan<D, MODE, kGroups, kPair>;
+    using Plan = SmemPlan<D, MODE, kGroups, kPair, kSplit>;
+    constexpr int kBN = Plan::kBN;                           // keys per tile
     constexpr bool kDoubleQ = Plan::kDoubleQ;
     constexpr int kFirstSoftmaxWarp = first_softmax_warp(kGroups);
     constexpr int kHalves = Plan::kHalves;
@@ -756,8 +766,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 
     // The warps of the first warpgroup need few registers (two of them are idle), the softmax warps hold a whole
     // row of scores and tangent scores each; the budgets are moved accordingly.
-    // (The forward-only softmax needs fewer registers than the 168 every thread of a 384-thread CTA starts with.)
-    constexpr bool kMoveRegs = kHasTQ;
+    // (The forward-only softmax with 64-key tiles needs fewer registers than the 168 every thread of a 384-thread CTA
+    // starts with; with 128-key tiles a thread holds 128 scores.)
+    constexpr bool kMoveRegs = kHasTQ || kBN > kBlockN;
     if (warp < kFirstSoftmaxWarp) {
     if (kMoveRegs) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsLightWarps));
     if (warp == kProducerWarp) {
@@ -810,7 +821,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     constexpr uint32_t kTxPerCta = (kHasTKV ? 2 * Plan::kKvHalfBytes : 0) + Plan::kKvHalfBytes;
                     constexpr uint32_t kRows32Off = kHasTKV ? kPairRegionB : 0;
                     if (lead_cta) mbar_arrive_expect_tx(smem_u32(&bar_slot_full[slot]), 2 * kTxPerCta);
-                    const int row0 = (w.tile0 + j) * kBlockN;
+                    const int row0 = (w.tile0 + j) * kBN;
 #pragma unroll
                     for (int hf = 0; hf < kHalves; ++hf) {
                         if (kHasTKV)
@@ -824,9 +835,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 // per 64-column half: [K_half (8 KB)][tK_half (8 KB)] so that [K ; tK] is one N = 128 operand
 #pragma unroll
                 for (int hf = 0; hf < kHalves; ++hf) {
-                    tma_load_4d(dst + hf * kKHalfStride, &tm_k, bar, hf * 64, w.h, (w.tile0 + j) * kBlockN, w.b);
+                    tma_load_4d(dst + hf * kKHalfStride, &tm_k, bar, hf * 64, w.h, (w.tile0 + j) * kBN, w.b);
                     if (kHasTKV)
-                        tma_load_4d(dst + hf * kKHalfStride + Plan::kKvHalfBytes, &tm_tk, bar, hf * 64, w.h, (w.tile0 + j) * kBlockN, w.b);
+                        tma_load_4d(dst + hf * kKHalfStride + Plan::kKvHalfBytes, &tm_tk, bar, hf * 64, w.h, (w.tile0 + j) * kBN, w.b);
                 }
                 return true;
             };
@@ -841,7 +852,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     constexpr uint32_t kTxPerCta = (kHasTKV ? 2 * Plan::kKvHalfBytes : 0) + Plan::kKvHalfBytes;
                     constexpr uint32_t kAtomOff = kHasTKV ? kPairRegionB : 0;
                     if (lead_cta) mbar_arrive_expect_tx(smem_u32(&bar_slot_full[slot]), 2 * kTxPerCta);
-                    const int row0 = (w.tile0 + j) * kBlockN;
+                    const int row0 = (w.tile0 + j) * kBN;
                     if (kHasTKV) {
 #pragma unroll
                         for (int hf = 0; hf < kHalves; ++hf)
@@ -854,9 +865,9 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 // [V_half0][V_half1][tV_half0][tV_half1]: consecutive 64-wide N atoms of [V | tV]
 #pragma unroll
                 for (int hf = 0; hf < kHalves; ++hf) {
-                    tma_load_4d(dst + hf * Plan::kKvHalfBytes, &tm_v, bar, hf * 64, w.h, (w.tile0 + j) * kBlockN, w.b);
+                    tma_load_4d(dst + hf * Plan::kKvHalfBytes, &tm_v, bar, hf * 64, w.h, (w.tile0 + j) * kBN, w.b);
                     if (kHasTKV)
-                        tma_load_4d(dst + (kHalves + hf) * Plan::kKvHalfBytes, &tm_tv, bar, hf * 64, w.h, (w.tile0 + j) * kBlockN, w.b);
+                        tma_load_4d(dst + (kHalves + hf) * Plan::kKvHalfBytes, &tm_tv, bar, hf * 64, w.h, (w.tile0 + j) * kBN, w.b);
                 }
                 return true;
             };
@@ -1049,8 +1060,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         {
             // (CTA pair: M = 256, 128 rows in each CTA; N counts the columns of both CTAs' parts of the B operand)
             constexpr int kMmaM = kPair ? 2 * kBlockM : kBlockM;
-            constexpr uint32_t kIdescS1 = make_idesc(kHasTKV ? 2 * kBlockN : kBlockN, false, kMmaM);  // Q x [K;tK] or Q x K
-            constexpr uint32_t kIdescS2 = make_idesc(kBlockN, false, kMmaM);                          // tQ x K
+            constexpr uint32_t kIdescS1 = make_idesc(kHasTKV ? 2 * kBN : kBN, false, kMmaM);  // Q x [K;tK] or Q x K
+            constexpr uint32_t kIdescS2 = make_idesc(kBN, false, kMmaM);                          // tQ x K
             constexpr uint32_t kIdescPV = make_idesc(kHasTKV ? 2 * D : D, true, kMmaM);               // P~ x [V|tV] or P~ x V
             constexpr uint32_t kIdescHV = make_idesc(D, true, kMmaM);                                 // H~ x V
             constexpr uint32_t kVLbo = Plan::kKvHalfBytes;   // bytes between 64-wide N atoms of a V slot
@@ -1118,7 +1129,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 for (int k = 1; k < D / 16; ++k) mma_ss1(tm_s, qd(k), kd(k), kIdescS1);
             };
             auto issue_scores_b = [&](int g, int buf, int slot, bool last_of_item) {
-                const uint32_t tm_ts = tmem + kScoreCol0 + buf * kScoreBufStride + kBlockN;
+                const uint32_t tm_ts = tmem + kScoreCol0 + buf * kScoreBufStride + kBN;
                 if (kHasTQ) {
                     if (kHasTKV) mma_ss1(tm_ts, tqd(0), k2d(0), kIdescS2);
                     else mma_ss0(tm_ts, tqd(0), k2d(0), kIdescS2);
@@ -1136,15 +1147,15 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const uint32_t tm_p = tmem + kScoreCol0 + buf * kScoreBufStride;
                 if (leader) TRACE(3, g);          // MMA: about to issue value MMAs
 #pragma unroll
-                for (int k = 0; k < kBlockN / 16; ++k) {
+                for (int k = 0; k < kBN / 16; ++k) {
                     mma_tsx(tmem_o, tm_p + k * 8, vd(k), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
                 }
             };
             auto issue_values_h = [&](int j, int g, int buf, int slot) {
-                const uint32_t tm_h = tmem + kScoreCol0 + buf * kScoreBufStride + kBlockN;
+                const uint32_t tm_h = tmem + kScoreCol0 + buf * kScoreBufStride + kBN;
                 if (kHasTQ) {
 #pragma unroll
-                    for (int k = 0; k < kBlockN / 16; ++k) {
+                    for (int k = 0; k < kBN / 16; ++k) {
                         mma_tsx(tmem_t, tm_h + k * 8, v2d(k), kIdescHV, (kHasTKV || j > 0 || k > 0) ? 1u : 0u);
                     }
                 }
@@ -1366,17 +1377,17 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 if (trace_me && g < kTraceSteps) g_trace[5 + ((warp - kFirstSoftmaxWarp) & 3)][g] = clock64();     // softmax warp: scores seen ready
 #endif
                 const uint32_t tm_s = tmem + lane_base + kScoreCol0 + bsel * kScoreBufStride;
-                const uint32_t tm_ts = tm_s + kBlockN;
+                const uint32_t tm_ts = tm_s + kBN;
 
-                uint32_t sv[kBlockN];
-                uint32_t tv[kBlockN];
+                uint32_t sv[kBN];
+                uint32_t tv[kBN];
                 // S first; tS is fetched while the row maximum is formed
 #pragma unroll
-                for (int c0 = 0; c0 < kBlockN; c0 += 32) TMEM_LD32(tm_s + c0, sv, c0);
+                for (int c0 = 0; c0 < kBN; c0 += 32) TMEM_LD32(tm_s + c0, sv, c0);
                 if (kGroups == 1 || !kHasTQ) tc_wait_ld();
                 if (kHasTQ) {
 #pragma unroll
-                    for (int c0 = 0; c0 < kBlockN; c0 += 32) TMEM_LD32(tm_ts + c0, tv, c0);
+                    for (int c0 = 0; c0 < kBN; c0 += 32) TMEM_LD32(tm_ts + c0, tv, c0);
                 }
                 if (kGroups == 2 && kHasTQ) tc_wait_ld();      // (two groups hide the latency by themselves: one wait)
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
@@ -1384,11 +1395,11 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #endif
 
                 // keys past Lk (zero-filled by TMA) must not enter the softmax
-                const int valid = args.Lk - (w.tile0 + j) * kBlockN;
-                if (valid < kBlockN) {
+                const int valid = args.Lk - (w.tile0 + j) * kBN;
+                if (valid < kBN) {
                     const uint32_t masked = neg_scale ? 0x7F800000u : 0xFF800000u;   // -inf after scaling
 #pragma unroll
-                    for (int c = 0; c < kBlockN; ++c) if (c >= valid) sv[c] = masked;
+                    for (int c = 0; c < kBN; ++c) if (c >= valid) sv[c] = masked;
                 }
 
                 // rowmax(S_ij) (four independent chains), in the log2 domain
@@ -1397,10 +1408,10 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 for (int u = 0; u < 4; ++u) mx4[u] = __uint_as_float(sv[u]);
                 if (!neg_scale) {
 #pragma unroll
-                    for (int c = 4; c < kBlockN; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(sv[c]));
+                    for (int c = 4; c < kBN; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(sv[c]));
                 } else {
 #pragma unroll
-                    for (int c = 4; c < kBlockN; ++c) mx4[c & 3] = fminf(mx4[c & 3], __uint_as_float(sv[c]));
+                    for (int c = 4; c < kBN; ++c) mx4[c & 3] = fminf(mx4[c & 3], __uint_as_float(sv[c]));
                 }
                 float mx = neg_scale ? fminf(fminf(mx4[0], mx4[1]), fminf(mx4[2], mx4[3]))
                                      : fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
@@ -1434,8 +1445,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 auto centre_of_first_tile = [&]() {
                     float sm4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
 #pragma unroll
-                    for (int c = 0; c < kBlockN; ++c) sm4[c & 3] += __uint_as_float(tv[c]);
-                    const int n_valid = valid < kBlockN ? valid : kBlockN;
+                    for (int c = 0; c < kBN; ++c) sm4[c & 3] += __uint_as_float(tv[c]);
+                    const int n_valid = valid < kBN ? valid : kBN;
                     return sc * ((sm4[0] + sm4[1]) + (sm4[2] + sm4[3])) / static_cast<float>(n_valid);
                 };
                 if (kHasTQ && kGroups == 1) tc_wait_ld();      // tS is in registers
@@ -1490,8 +1501,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 const uint64_t negm = pack_f32x2(-m_ref, -m_ref);
                 const uint64_t scsc = pack_f32x2(sc, sc);
                 const uint64_t negshift = pack_f32x2(-ts_shift, -ts_shift);
-                uint32_t pk_p[kBlockN / 2];
-                uint32_t pk_h[kBlockN / 2];
+                uint32_t pk_p[kBN / 2];
+                uint32_t pk_h[kBN / 2];
                 float lsum, rsum = 0.0f;
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
                 if (trace_me && quarter == 0 && g < kTraceSteps) g_trace[24][g] = clock64();    // softmax: the pass over the columns begins
@@ -1503,7 +1514,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     uint64_t ls2[2] = {0ull, 0ull};     // (+0.0f, +0.0f)
                     uint64_t rs2[2] = {0ull, 0ull};
 #pragma unroll
-                    for (int c = 0; c < kBlockN; c += 2) {
+                    for (int c = 0; c < kBN; c += 2) {
                         float x0, x1;
                         unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), c1c1, negm), x0, x1);
                         const float p0 = ex2f(x0), p1 = ex2f(x1);
@@ -1535,7 +1546,8 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
                 if (trace_me && quarter == 0 && g < kTraceSteps) g_trace[25][g] = clock64();    // softmax: ... and ends
 #endif
-                TMEM_ST32(tm_s, pk_p, 0);
+#pragma unroll
+                for (int c0 = 0; c0 < kBN / 2; c0 += 32) TMEM_ST32(tm_s + c0, pk_p, c0);      // bf16: two keys per column
                 if (kHasTQ) TMEM_ST32(tm_ts, pk_h, 0);
 #if defined(ATTN_JVP_TRACE) && ATTN_JVP_TRACE >= 2
                 if (trace_me && quarter == 0 && g < kTraceSteps) g_trace[28][g] = clock64();    // softmax: P~, H~ stores issued

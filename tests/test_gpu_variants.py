@@ -53,6 +53,11 @@ def test_every_variant_against_the_oracle(aj, oracle, mode, shape):
             if groups == 1:
                 if ref is None:
                     ref = (o, to, lse)
+                elif mode == "fwd":
+                    # the forward-only kernel takes 128 keys per tile on one CTA and 64 in the pair: another order
+                    # of summation, equal to one bf16 ulp
+                    assert (o.float() - ref[0].float()).abs().max().item() <= 2.0 ** -7 * ref[0].float().abs().max().item()
+                    assert (lse - ref[2]).abs().max().item() <= 1e-5
                 else:   # same arithmetic, same order: the CTA pair only changes who issues the MMAs
                     assert torch.equal(o, ref[0]) and torch.equal(lse, ref[2])
                     assert to is None or torch.equal(to, ref[1])
