@@ -130,12 +130,12 @@ struct KernelArgs {
 //   Two Q/tQ buffers (the variants that leave room: no K/V tangents, or D = 64): the next item's Q, tQ are loaded
 //   while the current item runs, ring slots hold exactly what the mode loads, and an item's output tiles are staged
 //   in its own Q/tQ buffer (dead once its last value MMAs are complete) instead of in ring slots.
-// ... except in the forward-only mode at D = 128 (one CTA per query tile, no key chunks), which takes 128 keys per
+// ... except in the forward-only mode (one CTA per query tile, no key chunks), which takes 128 keys per
 // tile: there is no tS, so a score buffer of 128 tensor-memory columns holds S of 128 keys, the N = 128 score MMAs
 // run at the pipe's full rate (64 cycles for twice the work of an N = 64 one at 54), and the per-tile costs of
 // the issuing and softmax warps (barriers, tensor-memory round trips, bookkeeping) are paid half as often.
 __host__ __device__ constexpr int key_tile(int D, int mode, bool split, bool pair) {
-    return (mode == kModeFwdOnly && D == 128 && !split && !pair) ? 2 * kBlockN : kBlockN;
+    return (mode == kModeFwdOnly && !split && !pair) ? 2 * kBlockN : kBlockN;
 }
 
 template <int D, int MODE, int kGroups, bool kPair, bool kSplit = false>
