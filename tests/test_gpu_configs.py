@@ -88,3 +88,20 @@ def test_full_size_workload(aj, oracle, name, n_rand, full_tiles, heads_full):
             assert (lse[b, h, rr] - cl).abs().max().item() <= 1e-3 * (1 + cl.abs().max().item())
         assert worst_o <= 1.0 and worst_t <= 1.0, (b, h, worst_o, worst_t)
         assert worst_ro <= CHUNK_REL_L2 and worst_rt <= CHUNK_REL_L2, (b, h, worst_ro, worst_rt)
+
+
+@pytest.mark.parametrize("name", ["image_dit_2b", "video_dit_1p3b", "image_dit_d64"])
+def test_full_size_forward_only(aj, oracle, name):
+    """The plain forward of the same kernel (the denominator of the bench's JVP / forward ratio) at full size: it
+    runs on its own variant (128-key tiles, two softmax groups), so it gets its own oracle check on sampled rows
+    and is compared with the O and LSE of the JVP call (other variant, other rounding of P~: bf16-level agreement)."""
+    w = synth.WORKLOADS[name]
+    x = synth.make_workload(w)
+    g = U.to_gpu(x)
+    o, _, lse = U.run(aj, g, w.scale, fwd_only=True)
+    rows = synth.sample_rows(w.B, w.H, w.Lq, n_random_per_head=3, seed=12)
+    U.check_all(oracle, aj, x, w.B, w.H, w.Lq, w.Lk, w.D, w.scale, rows, o, None, lse)
+    oj, _, lsej = U.run(aj, g, w.scale)
+    assert (lse - lsej).abs().max().item() <= 1e-4
+    d = (o.float() - oj.float())
+    assert d.norm().item() <= 5e-3 * oj.float().norm().item()
