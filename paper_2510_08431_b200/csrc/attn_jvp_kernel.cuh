@@ -1,14 +1,14 @@
 // Attention-JVP forward kernel for sm_100a (Algorithm 2: FlashAttention-2 forward with JVP).
 //
 // One CTA owns a 128-row query tile of one (batch, head) and streams the keys in
-// tiles of 64; CTAs are persistent (one per SM) and walk the query tiles round-robin, so that the epilogue of
+// tiles of 64 (128 in the forward-only mode); CTAs are persistent (one per SM) and walk the query tiles round-robin, so that the epilogue of
 // one tile overlaps the loads and the first score MMAs of the next.  Roles (warp-specialised, 384 threads, laid
 // out by warpgroup so that each can have its own register budget):
 //   warp 0      MMA issuer: the whole warp runs the loop in lock step, one elected lane's tcgen05.mma take effect,
 //               with accumulators in tensor memory.
 //   warp 1      TMA producer: Q,tQ per query tile, K|tK and V|tV tiles into a shared-memory ring.  (Warps 2, 3 idle.)
 //   warps 4-7   softmax: thread (w, lane) owns query row 32*(w%4) + lane (its tensor-memory lane) and
-//               all 64 columns of every score tile.  Reads S and tS from tensor memory, keeps m, l, r
+//               all columns of every score tile.  Reads S and tS from tensor memory, keeps m, l, r
 //               (Algorithm 2 lines 10-12, 16) in registers, writes P~ and H~ = P~ . tS back to tensor
 //               memory as bf16 MMA operands, and rescales the accumulators when the running max moves.
 //   warps 8-11  a second softmax group on alternate key tiles, or (one group) the epilogue warps, which run
@@ -105,7 +105,7 @@ struct KernelArgs {
     float* lse;
     int* host_status;   // mapped pinned host word, receives the timeout code
     int H, Lq, Lk;
-    int n_kv_tiles;     // 64-key tiles in all of Lk
+    int n_kv_tiles;     // key tiles (of the kernel variant's size) in all of Lk
     float scale;        // s
     float scale_log2;   // s * log2(e)
     // optional side output: mu = rowsum(P . tS) = d(LSE) along the tangent, fp32 [B][H][Lq] (may be null)
@@ -1307,7 +1307,7 @@ attn_jvp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
         if (kMoveRegs) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmaxWarps));
         // =====================================================================================
         // Softmax warps.  Thread (warp w, lane) owns query row 32*(w%4) + lane (= its tensor-memory
-        // lane) and all 64 columns of every score tile.
+        // lane) and all columns of every score tile.
         //
         // With two groups, group (g & 1) takes key tile g (numbered over all items of the CTA, like the score
         // buffers), so that two tiles are in work at a time and each scheduler has two softmax warps to hide
